@@ -1,0 +1,363 @@
+"""Pins for the CPU oracle: every oracle function is checked against something
+other than itself -- values printed in the paper, closed forms, brute force in
+pure Python on tiny inputs, or an unrelated library routine."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dash_oracle as oc
+from paper_2604_18103_b200 import workloads as wl
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "theory_speedup_vs_len.txt")
+
+
+def _table():
+    rows = []
+    with open(GOLD) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            n, nh, r, s = line.split()
+            rows.append((int(n), int(nh), float(r), float(s)))
+    return rows
+
+
+# ----------------------------------------------------------------- Appendix A
+def test_keep_count_matches_paper_table():
+    for n, n_hat, _, _ in _table():
+        assert oc.keep_count(n, 0.667, 64, 32, mode=1) == n_hat
+
+
+def test_flops_model_matches_paper_table():
+    for n, n_hat, r_pct, s in _table():
+        r, sp = oc.flops_single_shot(n, n_hat, L=28, l_s=11, d=3584, m=18944)
+        assert round(100.0 * r, 2) == pytest.approx(r_pct, abs=0.0051)
+        assert round(sp, 2) == pytest.approx(s, abs=0.0051)
+
+
+def test_keep_count_eq3_and_main_text_speedup():
+    # Eq. 3 by hand
+    assert oc.keep_count(8192, 0.4) == 4915
+    assert oc.keep_count(131072, 0.8) == 26214
+    assert oc.keep_count(1024, 0.5) == 512
+    assert oc.keep_count(100, 0.0) == 100
+    # Sec. 3.4: l_s = floor(0.4 L), rho = 0.667, T = 16384 -> 1.83x
+    k = oc.keep_count(16384, 0.667)
+    _, s = oc.flops_single_shot(16384, k, 28, 11, 3584, 18944)
+    assert abs(s - 1.83) < 0.015
+
+
+def test_flops_per_layer_terms():
+    # A(n) = 4nd^2 + 2n^2 d + 2ndm, term by term
+    assert oc.flops_per_layer(1, 1, 0) == 4 + 2
+    assert oc.flops_per_layer(2, 3, 5) == 4 * 2 * 9 + 2 * 4 * 3 + 2 * 2 * 3 * 5
+
+
+# ----------------------------------------------------------------- delta-norm
+def test_delta_norm_closed_forms():
+    g = torch.Generator().manual_seed(1)
+    H = torch.randn(37, 96, generator=g, dtype=torch.float64)
+    c = torch.linspace(-2, 2, 37, dtype=torch.float64)
+    U = H * c[:, None]
+    r = oc.delta_norm(U, H)
+    assert np.allclose(r, np.abs(c.numpy()), rtol=1e-6)
+    assert np.all(oc.delta_norm(torch.zeros_like(H), H) == 0)
+    # one-hot rows: exact
+    U1 = torch.zeros(4, 96, dtype=torch.float64); H1 = torch.zeros(4, 96, dtype=torch.float64)
+    for t in range(4):
+        U1[t, t] = 3.0 * (t + 1); H1[t, 95 - t] = 4.0
+    assert np.array_equal(oc.delta_norm(U1, H1), np.float32([0.75, 1.5, 2.25, 3.0]))
+    # ABS is Eq. 2 itself; REL * ||H|| = ABS
+    a = oc.delta_norm(U, H, mode=oc.ABS)
+    hn = np.array([math.sqrt(sum(float(x) ** 2 for x in row)) for row in H])
+    assert np.allclose(a, r * hn, rtol=1e-6)
+    # permuting the hidden dimension changes nothing
+    p = torch.randperm(96, generator=g)
+    assert np.allclose(oc.delta_norm(U[:, p], H[:, p]), r, rtol=1e-6)
+    # zero denominator guarded by eps
+    assert np.isfinite(oc.delta_norm(torch.ones(1, 8), torch.zeros(1, 8), eps=1e-12)).all()
+
+
+def test_delta_norm_brute_force_bf16_inputs():
+    g = torch.Generator().manual_seed(2)
+    U = torch.randn(5, 40, generator=g).to(torch.bfloat16)
+    H = torch.randn(5, 40, generator=g).to(torch.bfloat16)
+    r = oc.delta_norm(U, H)
+    for t in range(5):
+        su = sum(float(x) ** 2 for x in U[t].float())
+        sh = sum(float(x) ** 2 for x in H[t].float())
+        assert r[t] == np.float32(math.sqrt(su) / math.sqrt(sh))
+
+
+# --------------------------------------------------------------------- select
+def test_select_threshold_and_topk_agree():
+    g = torch.Generator().manual_seed(3)
+    r = torch.rand(500, generator=g).numpy().astype(np.float32)
+    cu = np.array([0, 200, 200, 500], dtype=np.int32)      # middle sequence empty
+    Ks = [77, 0, 123]
+    m_k = oc.select(r, cu, oc.KEEP_COUNT, keep_counts=Ks)
+    assert [int(m_k[cu[s]:cu[s + 1]].sum()) for s in range(3)] == Ks
+    for s in (0, 2):
+        seg, ms = r[cu[s]:cu[s + 1]], m_k[cu[s]:cu[s + 1]]
+        assert seg[ms == 1].min() > seg[ms == 0].max()           # keeps HIGH delta
+        tau = oc.kth_largest(seg, Ks[s])
+        m_t = oc.select(seg, np.array([0, seg.size], dtype=np.int32), oc.THRESHOLD, tau=tau)
+        assert np.array_equal(m_t, ms)
+    # rho = 0 keeps all
+    assert oc.select(r, cu, oc.KEEP_COUNT, keep_counts=[200, 0, 300]).all()
+
+
+def test_select_brute_force_tiny_and_ties():
+    r = np.float32([0.5, 0.1, 0.5, 0.9, 0.5, 0.2])
+    cu = np.array([0, 6], dtype=np.int32)
+    # K=3: 0.9 and the two lowest-index 0.5s
+    assert oc.select(r, cu, oc.KEEP_COUNT, keep_counts=[3]).tolist() == [1, 0, 1, 1, 0, 0]
+    assert oc.select(r, cu, oc.KEEP_COUNT, keep_counts=[1]).tolist() == [0, 0, 0, 1, 0, 0]
+    # threshold: halt iff r < tau (equality stays)
+    assert oc.select(r, cu, oc.THRESHOLD, tau=0.5).tolist() == [1, 0, 1, 1, 1, 0]
+    # NaN: stays under threshold, ranks first under top-K
+    rn = np.float32([0.5, np.nan, 0.7])
+    c3 = np.array([0, 3], dtype=np.int32)
+    assert oc.select(rn, c3, oc.THRESHOLD, tau=0.6).tolist() == [0, 1, 1]
+    assert oc.select(rn, c3, oc.KEEP_COUNT, keep_counts=[1]).tolist() == [0, 1, 0]
+
+
+def test_select_protected_prefix_suffix():
+    r = np.float32([0.0, 0.0, 0.9, 0.8, 0.7, 0.6, 0.0, 0.0])
+    cu = np.array([0, 8], dtype=np.int32)
+    # 2 first + 2 last protected although their score is lowest; K counts them
+    m = oc.select(r, cu, oc.KEEP_COUNT, keep_counts=[6], keep_first=2, keep_last=2)
+    assert m.tolist() == [1, 1, 1, 1, 0, 0, 1, 1]
+    m = oc.select(r, cu, oc.THRESHOLD, tau=0.75, keep_first=2, keep_last=2)
+    assert m.tolist() == [1, 1, 1, 1, 0, 0, 1, 1]
+    # K below the protected count: only the protected stay
+    m = oc.select(r, cu, oc.KEEP_COUNT, keep_counts=[1], keep_first=2, keep_last=2)
+    assert m.tolist() == [1, 1, 0, 0, 0, 0, 1, 1]
+    # kept length of Appendix A is met exactly
+    n = 1000
+    rr = np.random.default_rng(0).random(n).astype(np.float32)
+    K = oc.keep_count(n, 0.667, 64, 32, mode=1)
+    mm = oc.select(rr, np.array([0, n], dtype=np.int32), oc.KEEP_COUNT, keep_counts=[K], keep_first=64, keep_last=32)
+    assert int(mm.sum()) == K and mm[:64].all() and mm[-32:].all()
+
+
+# ------------------------------------------------------------ compact/scatter
+def test_compact_invariants_and_scatter_roundtrip():
+    n, d = 300, 16
+    mask = wl.random_mask(n, 0.4, seed=5)
+    cu = torch.tensor([0, 100, 100, 260, 300], dtype=torch.int32)
+    X = torch.randn(n, d, generator=torch.Generator().manual_seed(5)).to(torch.bfloat16)
+    pos = wl.positions(cu)
+    tok = torch.arange(n, dtype=torch.int32) + 1000
+    out = oc.compact(mask, cu, rows=[X], pos_in=pos, tok_in=tok)
+    idx = out["idx"]
+    assert out["n_out"] == int(mask.sum()) == idx.shape[0]            # popcount
+    assert np.all(np.diff(idx) > 0)                                   # stable / increasing
+    assert np.array_equal(idx, np.flatnonzero(mask.numpy()))
+    for s in range(4):
+        assert out["cu_out"][s + 1] - out["cu_out"][s] == int(mask[cu[s]:cu[s + 1]].sum())
+    assert torch.equal(out["rows"][0], X[mask.bool()])                # bit-exact rows
+    assert np.array_equal(out["pos_out"], pos.numpy()[idx])
+    assert np.array_equal(out["tok_out"], idx + 1000)
+    # scatter of the compacted rows back = identity on the active rows, others untouched
+    full = torch.full((n, d), -7.0, dtype=torch.bfloat16)
+    oc.scatter(out["rows"][0], idx, None, 2, full)
+    assert torch.equal(full[mask.bool()], X[mask.bool()])
+    assert (full[~mask.bool()] == -7.0).all()
+    # which = 0: only halted rows of the entry set are written
+    full2 = torch.zeros(n, d, dtype=torch.bfloat16)
+    oc.scatter(X, torch.arange(n, dtype=torch.int32), mask, 0, full2)
+    assert torch.equal(full2[~mask.bool()], X[~mask.bool()]) and (full2[mask.bool()] == 0).all()
+
+
+def test_compact_keep_all_and_keep_none():
+    n = 50
+    cu = torch.tensor([0, 20, 50], dtype=torch.int32)
+    X = torch.arange(n * 3, dtype=torch.float32).reshape(n, 3)
+    out = oc.compact(torch.ones(n, dtype=torch.uint8), cu, rows=[X])
+    assert torch.equal(out["rows"][0], X) and np.array_equal(out["cu_out"], cu.numpy())
+    out = oc.compact(torch.zeros(n, dtype=torch.uint8), cu, rows=[X])
+    assert out["n_out"] == 0 and out["rows"][0].shape[0] == 0 and not out["cu_out"].any()
+    out = oc.compact(torch.zeros(0, dtype=torch.uint8), torch.tensor([0, 0], dtype=torch.int32))
+    assert out["n_out"] == 0
+
+
+# ------------------------------------------------------------------ attention
+def _py_attention(Q, K, V, cu, scale):
+    """Independent brute force in pure Python floats."""
+    n, Hq, D = Q.shape
+    Hkv = K.shape[1]
+    G = Hq // Hkv
+    O = np.zeros((n, Hq, D))
+    for s in range(len(cu) - 1):
+        for i in range(cu[s], cu[s + 1]):
+            for h in range(Hq):
+                kv = h // G
+                sc = [scale * sum(float(Q[i, h, c]) * float(K[j, kv, c]) for c in range(D)) for j in range(cu[s], i + 1)]
+                m = max(sc)
+                e = [math.exp(x - m) for x in sc]
+                z = sum(e)
+                for c in range(D):
+                    O[i, h, c] = sum(e[jj] / z * float(V[cu[s] + jj, kv, c]) for jj in range(len(sc)))
+    return O
+
+
+def test_attention_tiny_brute_force():
+    g = torch.Generator().manual_seed(7)
+    cu = [0, 5, 5, 12]
+    Q = torch.randn(12, 4, 8, generator=g, dtype=torch.float64)
+    K = torch.randn(12, 2, 8, generator=g, dtype=torch.float64)
+    V = torch.randn(12, 2, 8, generator=g, dtype=torch.float64)
+    O, lse = oc.attention(Q, K, V, np.array(cu, dtype=np.int32), scale=0.3)
+    ref = _py_attention(Q.numpy(), K.numpy(), V.numpy(), cu, 0.3)
+    assert np.allclose(O, ref, rtol=1e-12, atol=1e-13)
+
+
+def test_attention_closed_forms():
+    g = torch.Generator().manual_seed(8)
+    n, Hq, Hkv, D = 40, 6, 2, 16
+    cu = np.array([0, 13, 40], dtype=np.int32)
+    Q = torch.randn(n, Hq, D, generator=g, dtype=torch.float64)
+    K = torch.randn(n, Hkv, D, generator=g, dtype=torch.float64)
+    V = torch.randn(n, Hkv, D, generator=g, dtype=torch.float64)
+    O, lse = oc.attention(Q, K, V, cu)
+    # first token of each sequence attends to itself only: O = v_0 of its kv head
+    for first in (0, 13):
+        for h in range(Hq):
+            assert np.allclose(O[first, h], V[first, h // 3].numpy(), atol=1e-14)
+            s00 = float((Q[first, h] * K[first, h // 3]).sum()) / math.sqrt(D)
+            assert abs(lse[first, h] - s00) < 1e-12
+    # V constant -> O is that constant
+    Vc = torch.ones_like(V) * 2.5
+    Oc, _ = oc.attention(Q, K, Vc, cu)
+    assert np.allclose(Oc, 2.5, atol=1e-13)
+    # Q = 0 -> uniform weights: O_i = prefix mean of v within the sequence
+    Oz, lz = oc.attention(torch.zeros_like(Q), K, V, cu)
+    for i in (0, 5, 12, 13, 39):
+        a = 0 if i < 13 else 13
+        for h in (0, 5):
+            assert np.allclose(Oz[i, h], V[a:i + 1, h // 3].mean(0).numpy(), atol=1e-13)
+            assert abs(lz[i, h] - math.log(i - a + 1)) < 1e-12
+    # sum_j exp(s_ij - lse_i) = 1
+    i, h = 30, 4
+    s = (K[13:31, h // 3] @ Q[i, h]) / math.sqrt(D)
+    assert abs(float(torch.exp(s - lse[i, h]).sum()) - 1.0) < 1e-12
+    # rows argument selects rows
+    Or, _ = oc.attention(Q, K, V, cu, rows=[39, 0, 13])
+    assert np.array_equal(Or, O[[39, 0, 13]])
+    # sequences are independent: swapping the two sequences permutes the outputs
+    perm = list(range(13, 40)) + list(range(0, 13))
+    Op, _ = oc.attention(Q[perm], K[perm], V[perm], np.array([0, 27, 40], dtype=np.int32))
+    assert np.allclose(Op, O[perm], atol=1e-13)
+
+
+def test_attention_matches_library_sdpa():
+    g = torch.Generator().manual_seed(9)
+    n, Hq, Hkv, D = 96, 8, 2, 32
+    Q = torch.randn(n, Hq, D, generator=g, dtype=torch.float64)
+    K = torch.randn(n, Hkv, D, generator=g, dtype=torch.float64)
+    V = torch.randn(n, Hkv, D, generator=g, dtype=torch.float64)
+    O, _ = oc.attention(Q, K, V, np.array([0, n], dtype=np.int32))
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        Q.transpose(0, 1)[None], K.transpose(0, 1).repeat_interleave(4, 0)[None],
+        V.transpose(0, 1).repeat_interleave(4, 0)[None], is_causal=True)[0].transpose(0, 1)
+    assert np.allclose(O, ref.numpy(), atol=1e-12)
+
+
+# ---------------------------------------------------------------------- glue
+def test_rmsnorm_and_rope_properties():
+    g = torch.Generator().manual_seed(10)
+    H = torch.randn(9, 64, generator=g, dtype=torch.float64)
+    y = oc.rmsnorm(H, torch.ones(64), eps=0.0)
+    assert np.allclose(np.mean(y * y, axis=1), 1.0)
+    assert np.allclose(oc.rmsnorm(3.0 * H, torch.ones(64), eps=0.0), y)
+    w = torch.linspace(0.5, 2.0, 64, dtype=torch.float64)
+    assert np.allclose(oc.rmsnorm(H, w, eps=0.0), y * w.numpy()[None])
+    # hand value: x = (3,4), mean sq = 12.5
+    assert np.allclose(oc.rmsnorm(torch.tensor([[3.0, 4.0]]), torch.ones(2), eps=0.0), [[3 / math.sqrt(12.5), 4 / math.sqrt(12.5)]])
+
+    X = torch.randn(7, 3, 16, generator=g, dtype=torch.float64)
+    pos = torch.tensor([0, 1, 2, 5, 11, 100, 4097])
+    R = oc.rope(X, pos, 10000.0)
+    assert np.allclose(R[0], X[0].numpy())                                   # pos 0: identity
+    assert np.allclose((R * R).sum(-1), (X * X).sum(-1).numpy())             # rotation keeps norms
+    # D = 2: plain 2-D rotation by pos radians
+    x2 = torch.tensor([[[1.0, 0.0]]])
+    assert np.allclose(oc.rope(x2, torch.tensor([2]), 10000.0), [[[math.cos(2), math.sin(2)]]])
+    # pair (i, i + D/2) with angle pos * base^(-2i/D): check one element by hand
+    i, D, p = 3, 16, 11
+    th = p * 10000.0 ** (-2 * i / D)
+    x = X[4, 1].numpy()
+    assert abs(R[4, 1, i] - (x[i] * math.cos(th) - x[i + 8] * math.sin(th))) < 1e-12
+    assert abs(R[4, 1, i + 8] - (x[i + 8] * math.cos(th) + x[i] * math.sin(th))) < 1e-12
+    # relative-position property: <R(q,m), R(k,n)> depends on m - n only
+    q = torch.randn(1, 1, 16, generator=g, dtype=torch.float64); k = torch.randn(1, 1, 16, generator=g, dtype=torch.float64)
+    d1 = (oc.rope(q, torch.tensor([9]), 1e4) * oc.rope(k, torch.tensor([4]), 1e4)).sum()
+    d2 = (oc.rope(q, torch.tensor([105]), 1e4) * oc.rope(k, torch.tensor([100]), 1e4)).sum()
+    assert abs(d1 - d2) < 1e-10
+
+
+def _torch_layer(H, W, pos, shape):
+    """Independent fp64 restatement of the block with torch library ops."""
+    Hd = H.double()
+    Hn = Hd * torch.rsqrt(Hd.pow(2).mean(-1, keepdim=True) + shape.rms_eps) * W["rms_w"].double()
+    n = Hd.shape[0]
+    q = (Hn @ W["Wq"].double()).view(n, shape.Hq, shape.D)
+    k = (Hn @ W["Wk"].double()).view(n, shape.Hkv, shape.D)
+    v = (Hn @ W["Wv"].double()).view(n, shape.Hkv, shape.D)
+    half = shape.D // 2
+    inv = shape.rope_base ** (-torch.arange(half, dtype=torch.float64) * 2 / shape.D)
+    ang = pos.double()[:, None] * inv[None]
+    cos, sin = torch.cat([ang.cos()] * 2, -1)[:, None], torch.cat([ang.sin()] * 2, -1)[:, None]
+    rot = lambda x: torch.cat([-x[..., half:], x[..., :half]], -1)
+    q, k = q * cos + rot(q) * sin, k * cos + rot(k) * sin
+    o = torch.nn.functional.scaled_dot_product_attention(
+        q.transpose(0, 1)[None], k.transpose(0, 1).repeat_interleave(shape.G, 0)[None],
+        v.transpose(0, 1).repeat_interleave(shape.G, 0)[None], is_causal=True)[0].transpose(0, 1)
+    U = o.reshape(n, -1) @ W["Wo"].double()
+    return U, Hd + U
+
+
+def test_layer_step_against_torch_restatement_and_rho0():
+    w = wl.config2(T=192, seed=11, shape=wl.MINI)
+    H, W = w.tensors["H"], w.weights[0]
+    pos = wl.positions(w.cu)
+    U_ref, Ht_ref = _torch_layer(H, W, pos, w.shape)
+    res = oc.layer_step(H, W, w.cu, pos, w.shape, tau=0.0)       # tau = 0: nothing halts
+    assert np.allclose(res["U"], U_ref.numpy(), rtol=1e-9, atol=1e-12)
+    assert np.allclose(res["Ht"], Ht_ref.numpy(), rtol=1e-9, atol=1e-12)
+    r_ref = (U_ref.norm(dim=1) / H.double().norm(dim=1)).float().numpy()
+    assert np.allclose(res["r"], r_ref, rtol=1e-6)
+    assert res["mask"].all() and res["n_out"] == 192                # rho = 0 == dense layer
+    assert np.array_equal(res["rows"][0], res["Ht"])
+    # halting at the median: K-th largest as threshold keeps exactly K
+    K = oc.keep_count(192, 0.5)
+    tau = oc.kth_largest(res["r"], K)
+    res2 = oc.layer_step(H, W, w.cu, pos, w.shape, tau=tau)
+    assert res2["n_out"] == K == int(res2["mask"].sum())
+    assert np.array_equal(res2["rows"][0], res2["Ht"][res2["mask"].astype(bool)])
+    # row-sampled evaluation equals the full one on those rows
+    res3 = oc.layer_step(H, W, w.cu, pos, w.shape, attn_rows=[0, 100, 191])
+    assert np.allclose(res3["U"], res["U"][[0, 100, 191]], rtol=1e-12, atol=1e-14)
+
+
+def test_workload_recipes_have_stated_structure():
+    w4 = wl.config4(T=4096, seed=3, shape=wl.MINI)
+    r = oc.delta_norm(w4.tensors["U"], w4.tensors["H"])
+    # relative delta ~ LogNormal(-3, 1): median near e^-3, heavy right tail
+    assert abs(math.log(float(np.median(r))) + 3.0) < 0.15
+    assert np.quantile(r, 0.99) / np.median(r) > 5
+    w5 = wl.config5(lengths=(512, 1024), seed=4, shape=wl.MINI, patch=64)
+    r5 = oc.delta_norm(w5.tensors["U"], w5.tensors["H"])
+    m5 = oc.select(r5, w5.cu, oc.THRESHOLD, tau=w5.tau)
+    img = w5.tensors["is_image"].numpy()
+    assert 0.80 < 1 - m5[img].mean() < 0.97          # about 90 % of image tokens halt
+    assert 0.03 < 1 - m5[~img].mean() < 0.20         # about 10 % of text tokens halt
+    assert int(img.sum()) == 384 + 768
+    # rank-8 structure of an image patch
+    Himg = w5.tensors["H"][:64].double()
+    sv = torch.linalg.svdvals(Himg)
+    assert sv[8] / sv[0] < 0.02
