@@ -1,0 +1,204 @@
+/*
+ * dash.h -- C ABI of the B200 (sm_100a) halted-prefill library.
+ *
+ * The library implements, for one Transformer block during prefill, the hot
+ * path of DASH (Delta Attention Selective Halting): the token-wise
+ * delta-attention score, the halting rule, the order-preserving compaction of
+ * the still-active tokens (with the frozen states of halted tokens written back
+ * to the full-length output), and causal grouped-query attention over the
+ * compacted active set.
+ *
+ * Conventions that hold for every entry point
+ *  - Every function returns an int status (DASH_OK = 0 or a DASH_ERR_* code).
+ *    Nothing throws, aborts or traps; invalid arguments are rejected before
+ *    any kernel is launched.
+ *  - Unless a parameter says "host", tensor pointers are DEVICE pointers owned
+ *    by the caller; they must stay valid until the work enqueued on `stream`
+ *    has finished.  The library allocates no device memory: scratch comes from
+ *    the caller's `ws` (size from dash_workspace_bytes), 256-byte aligned.
+ *  - `stream` is a cudaStream_t passed as void*.  All work is enqueued
+ *    asynchronously; no call synchronises except dash_check_status.
+ *  - Data-dependent sizes (number of active tokens, new sequence boundaries)
+ *    are written to device memory; the caller sizes outputs for the upper
+ *    bound it passes (`n`, the number of rows allocated).  Where a
+ *    `cu_seqlens` array is given, the true row count is cu_seqlens[S] (read on
+ *    the device) and rows at or beyond it are neither read nor written.
+ *  - Row-major tensors; `ld*` are row strides in ELEMENTS, `*_ld_bytes` in
+ *    bytes.  Data pointers and row strides must be multiples of 16 bytes.
+ *  - Kernels that wait (tile look-back, TMA/MMA barriers) give up after a
+ *    bounded number of polls and set DASH_ERR_TIMEOUT in a device status word
+ *    that dash_check_status returns.
+ */
+#ifndef DASH_H_
+#define DASH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DASH_OK               0
+#define DASH_ERR_INVALID_ARG  1
+#define DASH_ERR_UNSUPPORTED  2
+#define DASH_ERR_WORKSPACE    3
+#define DASH_ERR_CUDA         4
+#define DASH_ERR_TIMEOUT      5
+
+typedef enum { DASH_F32 = 0, DASH_BF16 = 1 } dash_dtype;
+/* REL: ||U_t|| / ||H_t|| (the "relative" delta-attention of Fig. 1);
+ * ABS: ||U_t||           (Eq. 2). */
+typedef enum { DASH_NORM_REL = 0, DASH_NORM_ABS = 1 } dash_norm_mode;
+typedef enum { DASH_SEL_THRESHOLD = 0, DASH_SEL_KEEP_COUNT = 1 } dash_sel_mode;
+
+#define DASH_MAX_ROW_STREAMS 8
+
+const char* dash_status_string(int status);
+
+/* Synchronises `stream`, returns the device status word (DASH_OK or
+ * DASH_ERR_TIMEOUT) and clears it. */
+int dash_check_status(void* stream);
+
+/* ---- host helpers (pure, no device work) --------------------------------
+ * Kept length.  mode 0: Eq. 3, K = floor((1 - rho) * n).
+ * mode 1: Appendix A: the first keep_first and last keep_last tokens always
+ * stay and floor(round(rho * (n - keep_first - keep_last))) of the others are
+ * dropped (round = to nearest, ties to even).  Returns -1 on invalid input. */
+int64_t dash_keep_count(int64_t n, double rho, int keep_first, int keep_last, int mode);
+/* Appendix A FLOPs proxy of one block: A(n) = 4 n d^2 + 2 n^2 d + 2 n d m. */
+double dash_flops_per_layer(double n, double d, double m);
+/* Appendix A: C_full / C_ours with C_full = L A(n), C_ours = l_s A(n) + (L - l_s) A(n_hat). */
+double dash_flops_speedup(double n, double n_hat, int L, int l_s, double d, double m);
+
+/* ---- step 1: delta-attention score (Eq. 1-2; Fig. 1 "relative") ----------
+ * Optional halting rule fused into the same pass (step 2, THRESHOLD mode):
+ * a token halts iff r_t < tau and it is not among the first keep_first / last
+ * keep_last tokens of its sequence (Appendix A). */
+typedef struct {
+    float          tau;
+    int            keep_first, keep_last;
+    const int32_t* cu_seqlens;   /* device [S+1] */
+    int            S;
+    uint8_t*       mask_out;     /* device [n], 1 = stays active */
+} dash_threshold;
+
+/* r_out[t] = ||U_t||_2 / max(||H_t||_2, eps)  (REL)  or  ||U_t||_2  (ABS), fp32
+ * accumulation.  U, H: [n, d] of type dt, d % 8 == 0.  If Hres_out != NULL the
+ * residual update H~_t = H_t + U_t (Preliminaries) is written in the same pass
+ * (may alias H).  If res_index != NULL (device int32 [n]), row t of the
+ * residual is written to row res_index[t] of Hres_out instead of row t.
+ * fused: NULL, or the threshold rule above.  n_dev: NULL, or a device int32
+ * holding the true row count (<= n). */
+int dash_delta_norm(const void* U, const void* H, int64_t n, int d, int64_t ldU, int64_t ldH,
+                    dash_dtype dt, dash_norm_mode mode, float eps, float* r_out,
+                    void* Hres_out, int64_t ldHres, const int32_t* res_index,
+                    const dash_threshold* fused, const int32_t* n_dev, void* stream);
+
+/* ---- step 2: halting rule (Eq. 3; Appendix A protected prefix/suffix) -----
+ * THRESHOLD: mask[t] = protected(t) || !(r[t] < tau)   (NaN stays active).
+ * KEEP_COUNT: per sequence s, keep_counts[s] (device int32 [S]) tokens stay in
+ *   total: the protected ones plus the largest scores of the others; ties at
+ *   the cut are broken toward the lower index; NaN ranks as +inf.
+ * r: device fp32 [n]; cu_seqlens: device int32 [S+1] over the current packed
+ * order; mask_out: device u8 [n] (1 = stays active). */
+int dash_select(const float* r, int64_t n, const int32_t* cu_seqlens, int S,
+                dash_sel_mode mode, float tau, const int32_t* keep_counts,
+                int keep_first, int keep_last, uint8_t* mask_out,
+                void* ws, size_t ws_bytes, void* stream);
+
+/* ---- step 3: compaction / scatter (Sec. 3.4; Alg. 1 "gathering tokens") ---
+ * One row tensor moved by the scan: dst[k] = src[idx[k]], rows of row_bytes
+ * (multiple of 4; 16-byte vector path when pointers, strides and row_bytes
+ * allow it). */
+typedef struct {
+    const void* src;
+    void*       dst;
+    int64_t     row_bytes, src_ld_bytes, dst_ld_bytes;
+} dash_rows;
+
+/* Exclusive prefix sum of mask (single pass, decoupled look-back) and stable
+ * gather of the active rows.  Outputs (device): idx_out[k] = source row of
+ * output row k (int32 [n]); cu_out int32 [S+1] = new packed boundaries;
+ * n_out_dev int32 = number of active rows (= cu_out[S]).  pos / tok (int32 per
+ * row: rotary position, row in the full-length buffer) are gathered when both
+ * the _in and _out pointer are non-NULL.  Any of idx_out, rows, pos, tok may be
+ * absent.  ws: dash_workspace_bytes(DASH_WS_COMPACT, n, S, ...). */
+int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
+                 const dash_rows* rows /*host array*/, int n_rows,
+                 const int32_t* pos_in, int32_t* pos_out,
+                 const int32_t* tok_in, int32_t* tok_out,
+                 int32_t* idx_out, int32_t* cu_out, int32_t* n_out_dev,
+                 void* ws, size_t ws_bytes, void* stream);
+
+/* dst_full[tok_index[i]] = src[i] for every i < n with sel[i] == which
+ * (which: 0 halted rows, 1 active rows, 2 every row; sel may be NULL for 2).
+ * tok_index NULL means the identity.  n_dev: NULL or device true row count. */
+int dash_scatter(const void* src, int64_t n, int64_t row_bytes, int64_t src_ld_bytes,
+                 const int32_t* tok_index, const uint8_t* sel, int which, const int32_t* n_dev,
+                 void* dst_full, int64_t dst_ld_bytes, void* stream);
+
+/* ---- step 4: causal GQA attention over the packed active set -------------
+ * For sequence s, query head h, packed row i in [cu[s], cu[s+1]):
+ *   O[i,h,:] = sum_{cu[s] <= j <= i} softmax_j(scale * q_i . k_j) v_j,
+ * key/value head h / (Hq / Hkv).  Only tokens present in the packed buffers
+ * own keys/values (halted tokens contribute none; Sec. 3.4).
+ * Q [n,Hq,D], O [n,Hq,D], K,V [n,Hkv,D] of type dt with row strides ldq, ldo,
+ * ldk, ldv (elements).  bf16 tensor-core math with fp32 accumulation and fp32
+ * softmax; DASH_F32 tensors are converted to bf16 on the way in (needs ws).
+ * lse: NULL or fp32 [Hq, n] = log-sum-exp of the scaled scores.
+ * D in {64, 128}; Hq % Hkv == 0; causal must be 1.  n: rows allocated;
+ * max_seqlen: upper bound of the longest sequence (grid sizing). */
+int dash_varlen_attention(const void* Q, const void* K, const void* V, void* O, float* lse,
+                          int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                          const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen,
+                          int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
+                          void* ws, size_t ws_bytes, void* stream);
+
+/* ---- the whole block step (Alg. 1, loop body without the FFN) ------------ */
+typedef struct {
+    int          d, Hq, Hkv, D;
+    dash_dtype   dt;               /* type of H, weights, x_full, H_next */
+    const void*  Wqkv;             /* [d, (Hq + 2 Hkv) D]: columns = Wq | Wk | Wv */
+    const void*  Wo;               /* [Hq D, d] */
+    const void*  rms_weight;       /* [d] */
+    float        rms_eps;
+    double       rope_base;
+    dash_norm_mode norm_mode;
+    float        norm_eps;
+    dash_sel_mode  sel_mode;
+    float        tau;              /* THRESHOLD */
+    const int32_t* keep_counts;    /* KEEP_COUNT: device int32 [S] */
+    int          keep_first, keep_last;
+    int          scatter_which;    /* rows of H~ written to x_full: 0 halted, 2 all */
+} dash_layer_cfg;
+
+/* Byte offsets of the intermediates inside the workspace of dash_layer_step
+ * (for inspection by tests and tools). */
+typedef struct {
+    size_t Hn, QKV, O, U, Ht, scratch, total;
+} dash_layer_ws_layout;
+int dash_layer_workspace(const dash_layer_cfg* cfg, int64_t n, int S, dash_layer_ws_layout* out);
+
+/* H_in [n, d]: packed hidden states of the tokens entering the block, with
+ * tok_index_in (row in the full-length buffer), pos_in (rotary position) and
+ * cu_in [S+1] (device).  Runs RMSNorm -> QKV projection -> rotary embedding ->
+ * causal attention -> output projection U -> r, H~ = H + U -> halting rule ->
+ * scatter of H~ into x_full [T, d] -> compaction of the tokens that stay
+ * active into H_next / tok_index_next / pos_next / cu_next / n_next_dev.
+ * r_out fp32 [n], mask_out u8 [n].  No host synchronisation. */
+int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, const int32_t* tok_index_in,
+                    const int32_t* pos_in, const int32_t* cu_in, int S, int64_t n, int64_t max_seqlen,
+                    void* x_full, void* H_next, int32_t* tok_index_next, int32_t* pos_next,
+                    int32_t* cu_next, int32_t* n_next_dev, float* r_out, uint8_t* mask_out,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/* ---- workspace sizes ------------------------------------------------------ */
+typedef enum { DASH_WS_SELECT = 0, DASH_WS_COMPACT = 1, DASH_WS_ATTENTION = 2 } dash_ws_op;
+/* n: rows allocated; S: sequences; Hq, Hkv, D, dt only matter for attention. */
+size_t dash_workspace_bytes(dash_ws_op op, int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DASH_H_ */

@@ -1,0 +1,403 @@
+// Causal grouped-query attention over a packed (varlen) batch of active tokens,
+// on tcgen05 tensor cores with TMEM accumulators, operands staged by TMA.
+//
+// Work unit (one CTA): 128 consecutive query rows of one head of one sequence.
+// Thread roles: warps 0-3 own one query row each (TMEM lane = row) and do the
+// online softmax; warp 4 allocates TMEM and its lane 0 issues every TMA load and
+// every tcgen05.mma.  Two CTAs share an SM (256 TMEM columns and < 113 KB of
+// shared memory each), so one CTA's softmax overlaps the other's MMAs.
+//
+// Per key block j (128 keys), with S and P aliasing the same TMEM columns:
+//   S = Q K_j^T  (SS MMA, fp32 in TMEM)  ->  softmax warps: mask, running max,
+//   exp2, row sum, P (bf16) back into TMEM, rescale O if the max moved  ->
+//   O += P V_j  (TS MMA: A operand read from TMEM)
+// Causal tile skipping: a query tile only visits key blocks 0..its own index.
+#include <math.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace dash {
+
+using namespace ptx;
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+int make_map_rows_heads(CUtensorMap* map, const void* base, int64_t rows, int heads, int D, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return DASH_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)heads, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)ld * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DASH_OK : DASH_ERR_CUDA;
+}
+
+int make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return DASH_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DASH_OK : DASH_ERR_CUDA;
+}
+
+constexpr int kBM = 128;                 // query rows per CTA
+constexpr int kBN = 128;                 // keys per block
+constexpr int kAttnThreads = 160;
+constexpr long long kWaitCycles = 4000000000LL;   // ~2 s: a wait that long is reported, not retried
+constexpr uint32_t kTmemCols = 256;
+
+struct AttnParams {
+    const int32_t* cu;
+    int S, Hq, Hkv, n_qtiles;
+    float scale_log2;       // softmax scale * log2(e)
+    float scale;
+    void* O;
+    int64_t ldo;            // elements
+    float* lse;             // [Hq, n] or null
+    int64_t n;
+    int* status;
+};
+
+template <int D>
+struct AttnSmem {
+    static constexpr int kTileBytes = kBM * D * 2;
+    static constexpr int kQ = 0, kK = kTileBytes, kV = 2 * kTileBytes, kBars = 3 * kTileBytes;
+    static constexpr int kTotal = kBars + 128;
+};
+
+template <int D, bool OUT_F32>
+__global__ void __launch_bounds__(kAttnThreads, 2)
+attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                 const __grid_constant__ CUtensorMap mapV, const AttnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    using L = AttnSmem<D>;
+    constexpr int KCH = D / 64;              // 64-element (128-byte) chunks along D
+    constexpr int kChunkBytes = kBM * 128;   // one chunk: 128 rows x 128 B
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base + L::kQ, sK = smem_base + L::kK, sV = smem_base + L::kV;
+    const uint32_t bars = smem_base + L::kBars;
+    const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_o = bars + 32, bar_p = bars + 40;
+    const uint32_t tmem_slot = bars + 64;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 64);
+    volatile uint32_t* abort_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 68);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // heavy (late) query tiles first; the heads of one KV group run together
+    const int per_tile = p.Hq * p.S;
+    const int qt = p.n_qtiles - 1 - (int)(blockIdx.x / per_tile);
+    const int rem = (int)(blockIdx.x % per_tile);
+    const int h = rem % p.Hq, s = rem / p.Hq;
+    const int kvh = h / (p.Hq / p.Hkv);
+    const int seq_a = p.cu[s], seq_b = p.cu[s + 1];
+    const int len = seq_b - seq_a;
+    const int q0 = qt * kBM;
+    if (q0 >= len) return;                                   // uniform for the CTA: nothing allocated yet
+    const int nblk = qt + 1;                                 // causal: key blocks 0..qt
+
+    if (warp == 4) {
+        if (lane == 0) {
+            mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1);
+            mbar_init(bar_s, 1); mbar_init(bar_o, 1); mbar_init(bar_p, 128);
+            *abort_gen = 0;
+            fence_barrier_init();
+            fence_proxy_async_smem();
+            prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV);
+        }
+        __syncwarp();
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_gen;
+    const uint32_t tS = tmem, tP = tmem, tO = tmem + 128;
+
+    constexpr uint32_t idesc_s = idesc_bf16_f32(kBM, kBN, false, false);
+    constexpr uint32_t idesc_o = idesc_bf16_f32(kBM, D, false, true);
+
+    if (warp == 4) {
+        if (lane == 0) {
+            bool ok = true;
+            mbar_arrive_expect_tx(bar_q, L::kTileBytes);
+            for (int c = 0; c < KCH; ++c) tma_load_3d(sQ + c * kChunkBytes, &mapQ, bar_q, c * 64, h, seq_a + q0);
+            mbar_arrive_expect_tx(bar_k, L::kTileBytes);
+            for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, kvh, seq_a);
+            mbar_arrive_expect_tx(bar_v, L::kTileBytes);
+            for (int c = 0; c < KCH; ++c) tma_load_3d(sV + c * kChunkBytes, &mapV, bar_v, c * 64, kvh, seq_a);
+            ok = mbar_wait(bar_q, 0, kWaitCycles);
+            for (int j = 0; j < nblk && ok; ++j) {
+                const uint32_t ph = j & 1;
+                ok = ok && mbar_wait(bar_k, ph, kWaitCycles);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * kChunkBytes + (kk & 3) * 32;
+                    mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), idesc_s, kk > 0);
+                }
+                tc_commit(bar_s);
+                ok = mbar_wait(bar_s, ph, kWaitCycles);
+                if (!ok) break;
+                if (j + 1 < nblk) {
+                    mbar_arrive_expect_tx(bar_k, L::kTileBytes);
+                    for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, kvh, seq_a + (j + 1) * kBN);
+                }
+                ok = mbar_wait(bar_p, ph, kWaitCycles) && mbar_wait(bar_v, ph, kWaitCycles);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < kBN / 16; ++kk) {
+                    // P: 128 lanes x (16 keys = 8 packed columns) per step; V: 16 keys = two 8-row groups of 1 KB
+                    mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
+                }
+                tc_commit(bar_o);
+                ok = mbar_wait(bar_o, ph, kWaitCycles);
+                if (!ok) break;
+                if (j + 1 < nblk) {
+                    mbar_arrive_expect_tx(bar_v, L::kTileBytes);
+                    for (int c = 0; c < KCH; ++c) tma_load_3d(sV + c * kChunkBytes, &mapV, bar_v, c * 64, kvh, seq_a + (j + 1) * kBN);
+                }
+            }
+            if (!ok) { *abort_gen = 1; atomicExch(p.status, DASH_ERR_TIMEOUT); }
+        }
+    } else {
+        // ---- softmax warps: thread <-> query row ----
+        const int row = tid;                               // 0..127
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const bool row_valid = (q0 + row) < len;
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nblk; ++j) {
+            const uint32_t ph = j & 1;
+            ok = mbar_wait(bar_s, ph, kWaitCycles);
+            if (!ok || *abort_gen) { ok = false; break; }
+            tc_fence_after();
+            uint32_t sreg[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_base + c * 32, &sreg[c * 32]);
+            tmem_wait_ld();
+            const bool diag = (j == qt);
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 128; ++c) {
+                float v = __uint_as_float(sreg[c]);
+                if (diag && c > row) v = -INFINITY;
+                sreg[c] = __float_as_uint(v);
+                mx = fmaxf(mx, v);
+            }
+            const float m_new = fmaxf(m, mx);
+            const float msl = m_new * p.scale_log2;
+            const float alpha = ex2((m - m_new) * p.scale_log2);
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 128; c += 2) {
+                float p0 = ex2(fmaf(__uint_as_float(sreg[c]), p.scale_log2, -msl));
+                float p1 = ex2(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl));
+                sum += p0 + p1;
+                sreg[c >> 1] = pack_bf16(p0, p1);
+            }
+            l = l * alpha + sum;
+            m = m_new;
+            tmem_st32(tP + lane_base, &sreg[0]);
+            tmem_st32(tP + lane_base + 32, &sreg[32]);
+            if (j > 0) {
+                // O still holds the previous blocks' sum scaled by the old max
+                const bool need = __any_sync(0xffffffffu, alpha != 1.0f);
+                if (need) {
+                    ok = mbar_wait(bar_o, (j - 1) & 1, kWaitCycles);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + lane_base + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tmem_st32(tO + lane_base + c * 32, o);
+                    }
+                }
+            }
+            if (diag) {
+                // keys past the end of the sequence: their V rows may hold anything (another
+                // sequence, or never-written memory); zero them so 0 * garbage cannot make a NaN
+                ok = mbar_wait(bar_v, ph, kWaitCycles);
+                if (!ok) break;
+                if (j * kBN + row >= len) {
+#pragma unroll
+                    for (int c = 0; c < KCH; ++c) {
+                        uint4* rowp = reinterpret_cast<uint4*>(smem_gen + L::kV + c * kChunkBytes + row * 128);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) rowp[e] = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async_smem();
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p);
+        }
+        if (ok) ok = mbar_wait(bar_o, (nblk - 1) & 1, kWaitCycles);
+        if (ok && !*abort_gen) {
+            tc_fence_after();
+            const float inv = 1.0f / l;
+            const int64_t grow = (int64_t)seq_a + q0 + row;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tO + lane_base + c * 32, o);
+                tmem_wait_ld();
+                if (row_valid) {
+                    if (OUT_F32) {
+                        float* dst = reinterpret_cast<float*>(p.O) + grow * p.ldo + (int64_t)h * D + c * 32;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            uint4 v;
+                            v.x = __float_as_uint(__uint_as_float(o[e]) * inv); v.y = __float_as_uint(__uint_as_float(o[e + 1]) * inv);
+                            v.z = __float_as_uint(__uint_as_float(o[e + 2]) * inv); v.w = __float_as_uint(__uint_as_float(o[e + 3]) * inv);
+                            st_v4(dst + e, v);
+                        }
+                    } else {
+                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.O) + grow * p.ldo + (int64_t)h * D + c * 32;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            uint4 v;
+                            v.x = pack_bf16(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv);
+                            v.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+                            v.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
+                            v.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
+                            st_v4(dst + e, v);
+                        }
+                    }
+                }
+            }
+            if (row_valid && p.lse) p.lse[(int64_t)h * p.n + grow] = m * p.scale + logf(l);
+        } else if (!ok && lane == 0) {
+            atomicExch(p.status, DASH_ERR_TIMEOUT);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+__global__ void f32_to_bf16_rows_kernel(const float* __restrict__ src, int64_t ld_src, __nv_bfloat16* __restrict__ dst, int64_t ld_dst,
+                                        int64_t rows, int cols) {
+    const int64_t total = rows * (cols / 4);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t r = i / (cols / 4);
+        int c = (int)(i % (cols / 4)) * 4;
+        float4 v = *reinterpret_cast<const float4*>(src + r * ld_src + c);
+        uint2 o = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+        *reinterpret_cast<uint2*>(dst + r * ld_dst + c) = o;
+    }
+}
+
+size_t attention_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt) {
+    (void)S;
+    if (dt == DASH_BF16) return 256;
+    return align_up((size_t)n * (Hq + 2 * Hkv) * D * 2, 256) + 256;
+}
+
+template <int D, bool OUT_F32>
+static int launch_attention(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p, int grid, cudaStream_t st) {
+    using L = AttnSmem<D>;
+    const int smem = L::kTotal + 1024;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(attention_kernel<D, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
+        configured = true;
+    }
+    attention_kernel<D, OUT_F32><<<grid, kAttnThreads, smem, st>>>(mq, mk, mv, p);
+    return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+}
+
+}  // namespace dash
+
+using namespace dash;
+
+extern "C" int dash_varlen_attention(const void* Q, const void* K, const void* V, void* O, float* lse,
+                                     int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                                     const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen,
+                                     int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
+                                     void* ws, size_t ws_bytes, void* stream) {
+    if (n < 0 || S < 1 || max_seqlen < 0 || Hq < 1 || Hkv < 1 || !cu_seqlens) return DASH_ERR_INVALID_ARG;
+    if (dt != DASH_F32 && dt != DASH_BF16) return DASH_ERR_INVALID_ARG;
+    if (D != 64 && D != 128) return DASH_ERR_UNSUPPORTED;
+    if (Hq % Hkv) return DASH_ERR_INVALID_ARG;
+    if (causal != 1) return DASH_ERR_UNSUPPORTED;
+    if (n > 0x7fffffffLL || max_seqlen > n) return DASH_ERR_INVALID_ARG;
+    if (n == 0 || max_seqlen == 0) return DASH_OK;
+    if (!Q || !K || !V || !O) return DASH_ERR_INVALID_ARG;
+    const int es = (dt == DASH_BF16) ? 2 : 4;
+    if (ldq < (int64_t)Hq * D || ldo < (int64_t)Hq * D || ldk < (int64_t)Hkv * D || ldv < (int64_t)Hkv * D) return DASH_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return DASH_ERR_INVALID_ARG;
+    if ((ldq * es) % 16 || (ldk * es) % 16 || (ldv * es) % 16 || (ldo * es) % 16) return DASH_ERR_INVALID_ARG;
+    if (!(scale > 0.f)) return DASH_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    const void *q = Q, *k = K, *v = V;
+    int64_t lq = ldq, lk = ldk, lv = ldv;
+    if (dt == DASH_F32) {
+        if (!ws || ((uintptr_t)ws % 256) || ws_bytes < attention_ws_bytes(n, S, Hq, Hkv, D, dt)) return DASH_ERR_WORKSPACE;
+        __nv_bfloat16* qb = (__nv_bfloat16*)ws;
+        __nv_bfloat16* kb = qb + (size_t)n * Hq * D;
+        __nv_bfloat16* vb = kb + (size_t)n * Hkv * D;
+        const int cap = sm_count() * 8;
+        auto cvt = [&](const void* src, int64_t ld, __nv_bfloat16* dst, int cols) {
+            int64_t total = n * (cols / 4);
+            int grid = (int)((total + 255) / 256);
+            if (grid > cap) grid = cap;
+            f32_to_bf16_rows_kernel<<<grid, 256, 0, st>>>((const float*)src, ld, dst, cols, n, cols);
+        };
+        cvt(Q, ldq, qb, Hq * D); cvt(K, ldk, kb, Hkv * D); cvt(V, ldv, vb, Hkv * D);
+        DASH_CUDA_TRY(cudaGetLastError());
+        q = qb; k = kb; v = vb;
+        lq = (int64_t)Hq * D; lk = lv = (int64_t)Hkv * D;
+    }
+    CUtensorMap mq, mk, mv;
+    int rc;
+    if ((rc = make_map_rows_heads(&mq, q, n, Hq, D, lq, kBM)) != DASH_OK) return rc;
+    if ((rc = make_map_rows_heads(&mk, k, n, Hkv, D, lk, kBN)) != DASH_OK) return rc;
+    if ((rc = make_map_rows_heads(&mv, v, n, Hkv, D, lv, kBN)) != DASH_OK) return rc;
+
+    AttnParams p;
+    p.cu = cu_seqlens; p.S = S; p.Hq = Hq; p.Hkv = Hkv;
+    p.n_qtiles = (int)((max_seqlen + kBM - 1) / kBM);
+    p.scale = scale;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.O = O; p.ldo = ldo; p.lse = lse; p.n = n;
+    p.status = status_word_ptr();
+    if (!p.status) return DASH_ERR_CUDA;
+    const int64_t grid64 = (int64_t)p.n_qtiles * Hq * S;
+    if (grid64 > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
+    const int grid = (int)grid64;
+    if (D == 128) return dt == DASH_F32 ? launch_attention<128, true>(mq, mk, mv, p, grid, st) : launch_attention<128, false>(mq, mk, mv, p, grid, st);
+    return dt == DASH_F32 ? launch_attention<64, true>(mq, mk, mv, p, grid, st) : launch_attention<64, false>(mq, mk, mv, p, grid, st);
+}

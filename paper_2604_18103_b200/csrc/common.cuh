@@ -1,0 +1,91 @@
+// Shared host/device helpers of the library (no method arithmetic lives here).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dash.h"
+
+#define DASH_CUDA_TRY(expr)                          \
+    do {                                             \
+        cudaError_t e__ = (expr);                    \
+        if (e__ != cudaSuccess) return DASH_ERR_CUDA; \
+    } while (0)
+
+namespace dash {
+
+constexpr int kWarp = 32;
+// polls before a device-side wait gives up and records DASH_ERR_TIMEOUT
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+// Device address of the per-device status word (host side; one word per GPU).
+int* status_word_ptr();
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int sm_count() {
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms > 0 ? sms : 148;
+}
+
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_v4(void* p, uint4 v) {
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// streaming store: written once, not re-read by this kernel
+__device__ __forceinline__ void st_cs_v4(void* p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Copy one row of `bytes` (multiple of 16, 16-byte aligned ends) with a warp.
+__device__ __forceinline__ void warp_copy_row16(const char* __restrict__ src, char* __restrict__ dst, int64_t bytes, int lane) {
+    const int nvec = (int)(bytes >> 4);
+    for (int base = 0; base < nvec; base += 32 * 4) {
+        uint4 r[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            int v = base + k * 32 + lane;
+            if (v < nvec) r[k] = ld_nc_v4(src + ((int64_t)v << 4));
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            int v = base + k * 32 + lane;
+            if (v < nvec) st_v4(dst + ((int64_t)v << 4), r[k]);
+        }
+    }
+}
+// Same for rows that are only 4-byte granular.
+__device__ __forceinline__ void warp_copy_row4(const char* __restrict__ src, char* __restrict__ dst, int64_t bytes, int lane) {
+    const int nw = (int)(bytes >> 2);
+    for (int v = lane; v < nw; v += 32)
+        reinterpret_cast<uint32_t*>(dst)[v] = reinterpret_cast<const uint32_t*>(src)[v];
+}
+
+// sequence that holds packed row t: largest s with cu[s] <= t (skips empty sequences)
+__device__ __forceinline__ int find_seq(const int32_t* __restrict__ cu, int S, int t) {
+    int lo = 0, hi = S;   // invariant: cu[lo] <= t < cu[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (cu[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+}  // namespace dash

@@ -1,0 +1,524 @@
+// HBM-bound kernels of the halted-prefill path: delta-attention score (+ fused
+// residual and threshold), halting rule, single-pass compaction, scatter.
+#include "common.cuh"
+
+namespace dash {
+
+// ---------------------------------------------------------------------------
+// step 1: r_t = ||U_t|| / max(||H_t||, eps)   (Eq. 2; "relative" form of Fig. 1)
+// One warp per row, 128-bit loads, 8 loads in flight per lane, fp32 sums,
+// shuffle reduction.  Optional: H~ = H + U written in the same pass (optionally
+// to an indexed row), and the threshold rule applied to r.
+// ---------------------------------------------------------------------------
+struct FusedThreshold {
+    float tau;
+    int keep_first, keep_last;
+    const int32_t* cu;
+    int S;
+    uint8_t* mask_out;
+};
+
+template <bool BF16>
+__device__ __forceinline__ float sumsq_vec(uint4 v) {
+    if (BF16) {
+        float a0 = bf16lo(v.x), a1 = bf16hi(v.x), a2 = bf16lo(v.y), a3 = bf16hi(v.y);
+        float a4 = bf16lo(v.z), a5 = bf16hi(v.z), a6 = bf16lo(v.w), a7 = bf16hi(v.w);
+        return a0 * a0 + a1 * a1 + a2 * a2 + a3 * a3 + a4 * a4 + a5 * a5 + a6 * a6 + a7 * a7;
+    } else {
+        float a0 = __uint_as_float(v.x), a1 = __uint_as_float(v.y), a2 = __uint_as_float(v.z), a3 = __uint_as_float(v.w);
+        return a0 * a0 + a1 * a1 + a2 * a2 + a3 * a3;
+    }
+}
+template <bool BF16>
+__device__ __forceinline__ uint4 add_vec(uint4 a, uint4 b) {
+    uint4 o;
+    if (BF16) {
+        o.x = pack_bf16(bf16lo(a.x) + bf16lo(b.x), bf16hi(a.x) + bf16hi(b.x));
+        o.y = pack_bf16(bf16lo(a.y) + bf16lo(b.y), bf16hi(a.y) + bf16hi(b.y));
+        o.z = pack_bf16(bf16lo(a.z) + bf16lo(b.z), bf16hi(a.z) + bf16hi(b.z));
+        o.w = pack_bf16(bf16lo(a.w) + bf16lo(b.w), bf16hi(a.w) + bf16hi(b.w));
+    } else {
+        o.x = __float_as_uint(__uint_as_float(a.x) + __uint_as_float(b.x));
+        o.y = __float_as_uint(__uint_as_float(a.y) + __uint_as_float(b.y));
+        o.z = __float_as_uint(__uint_as_float(a.z) + __uint_as_float(b.z));
+        o.w = __float_as_uint(__uint_as_float(a.w) + __uint_as_float(b.w));
+    }
+    return o;
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(256)
+delta_norm_kernel(const char* __restrict__ U, const char* __restrict__ H, int64_t n, int nvec,
+                  int64_t ldU_b, int64_t ldH_b, int mode, float eps, float* __restrict__ r_out,
+                  char* Hres, int64_t ldR_b, const int32_t* __restrict__ res_index,
+                  FusedThreshold ft, const int32_t* __restrict__ n_dev) {
+    const int lane = threadIdx.x & 31;
+    const int wpb = blockDim.x >> 5;
+    if (n_dev) { int64_t nd = *n_dev; if (nd < n) n = nd; }
+    const bool need_h = (mode == DASH_NORM_REL) || (Hres != nullptr);
+    constexpr int CH = 4;
+    for (int64_t row = (int64_t)blockIdx.x * wpb + (threadIdx.x >> 5); row < n; row += (int64_t)gridDim.x * wpb) {
+        const char* u = U + row * ldU_b;
+        const char* h = H + row * ldH_b;
+        char* o = nullptr;
+        if (Hres) o = Hres + (res_index ? (int64_t)res_index[row] : row) * ldR_b;
+        float su = 0.f, sh = 0.f;
+        for (int base = 0; base < nvec; base += 32 * CH) {
+            uint4 a[CH], b[CH];
+#pragma unroll
+            for (int k = 0; k < CH; ++k) {
+                int v = base + k * 32 + lane;
+                if (v < nvec) {
+                    a[k] = ld_nc_v4(u + ((int64_t)v << 4));
+                    if (need_h) b[k] = ld_nc_v4(h + ((int64_t)v << 4));
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < CH; ++k) {
+                int v = base + k * 32 + lane;
+                if (v < nvec) {
+                    su += sumsq_vec<BF16>(a[k]);
+                    if (need_h) {
+                        sh += sumsq_vec<BF16>(b[k]);
+                        if (o) st_v4(o + ((int64_t)v << 4), add_vec<BF16>(a[k], b[k]));
+                    }
+                }
+            }
+        }
+        su = warp_sum(su);
+        sh = warp_sum(sh);
+        if (lane == 0) {
+            float num = sqrtf(su);
+            float r = (mode == DASH_NORM_ABS) ? num : num / fmaxf(sqrtf(sh), eps);
+            r_out[row] = r;
+            if (ft.mask_out) {
+                int s = find_seq(ft.cu, ft.S, (int)row);
+                int local = (int)row - ft.cu[s], len = ft.cu[s + 1] - ft.cu[s];
+                bool prot = (local < ft.keep_first) || (local >= len - ft.keep_last);
+                ft.mask_out[row] = (prot || !(r < ft.tau)) ? 1 : 0;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// step 2: halting rule
+// ---------------------------------------------------------------------------
+__global__ void select_threshold_kernel(const float* __restrict__ r, int64_t n, const int32_t* __restrict__ cu, int S,
+                                        float tau, int keep_first, int keep_last, uint8_t* __restrict__ mask) {
+    int64_t total = cu[S];
+    if (total < n) n = total;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < n; t += (int64_t)gridDim.x * blockDim.x) {
+        int s = find_seq(cu, S, (int)t);
+        int local = (int)t - cu[s], len = cu[s + 1] - cu[s];
+        bool prot = (local < keep_first) || (local >= len - keep_last);
+        mask[t] = (prot || !(r[t] < tau)) ? 1 : 0;
+    }
+}
+
+// monotone map fp32 -> u32 (larger value = larger key); NaN -> max; -0 -> +0
+__device__ __forceinline__ uint32_t order_key(float f) {
+    uint32_t b = __float_as_uint(f);
+    if ((b & 0x7fffffffu) > 0x7f800000u) return 0xffffffffu;
+    if (b == 0x80000000u) b = 0;
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// exclusive scan of one int per thread over a 1024-thread block; total returned to all
+__device__ __forceinline__ int block_excl_scan_1024(int v, int* s_warp, int* total) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) s_warp[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+        int x = s_warp[lane];
+        int xi = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, xi, o);
+            if (lane >= o) xi += t;
+        }
+        s_warp[lane] = xi - x;
+        if (lane == 31) s_warp[32] = xi;
+    }
+    __syncthreads();
+    int res = s_warp[w] + inc - v;
+    *total = s_warp[32];
+    __syncthreads();
+    return res;
+}
+
+// One 1024-thread CTA per sequence: 4-pass MSB radix select of the k-th largest
+// key among the eligible (unprotected) tokens, then one ordered pass that keeps
+// keys above the cut and the lowest-index ties.
+__global__ void __launch_bounds__(1024)
+select_keep_count_kernel(const float* __restrict__ r, const int32_t* __restrict__ cu, int S,
+                         const int32_t* __restrict__ keep_counts, int keep_first, int keep_last,
+                         uint8_t* __restrict__ mask) {
+    __shared__ int hist[256];
+    __shared__ int s_warp[33];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_remaining;
+    const int s = blockIdx.x;
+    const int a = cu[s], b = cu[s + 1], ns = b - a;
+    if (ns <= 0) return;
+    const int kf = min(max(keep_first, 0), ns);
+    const int kl = min(max(keep_last, 0), ns - kf);
+    const int e0 = a + kf, e1 = b - kl;          // eligible range [e0, e1)
+    const int n_el = e1 - e0;
+    int k_el = keep_counts[s] - (kf + kl);
+    k_el = min(max(k_el, 0), n_el);
+    for (int t = a + threadIdx.x; t < e0; t += blockDim.x) mask[t] = 1;
+    for (int t = e1 + threadIdx.x; t < b; t += blockDim.x) mask[t] = 1;
+    if (k_el == 0 || k_el == n_el) {
+        uint8_t v = k_el ? 1 : 0;
+        for (int t = e0 + threadIdx.x; t < e1; t += blockDim.x) mask[t] = v;
+        return;
+    }
+    uint32_t prefix = 0, pmask = 0;
+    int remaining = k_el;                         // rank (from the top) inside the current bucket
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+        for (int t = e0 + threadIdx.x; t < e1; t += blockDim.x) {
+            uint32_t key = order_key(r[t]);
+            if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int acc = 0, bsel = 0;
+            for (int bk = 255; bk >= 0; --bk) {
+                if (acc + hist[bk] >= remaining) { bsel = bk; break; }
+                acc += hist[bk];
+            }
+            s_prefix = prefix | ((uint32_t)bsel << shift);
+            s_remaining = remaining - acc;
+        }
+        __syncthreads();
+        prefix = s_prefix;
+        remaining = s_remaining;
+        pmask |= (0xffu << shift);
+        __syncthreads();
+    }
+    // prefix = key of the k-th largest; `remaining` of the tokens that tie with it stay
+    const uint32_t cut = prefix;
+    const int per = (n_el + blockDim.x - 1) / blockDim.x;
+    const int t0 = min(e0 + (int)threadIdx.x * per, e1), t1 = min(t0 + per, e1);
+    int ties = 0;
+    for (int t = t0; t < t1; ++t) ties += (order_key(r[t]) == cut);
+    int total;
+    int rank = block_excl_scan_1024(ties, s_warp, &total);
+    for (int t = t0; t < t1; ++t) {
+        uint32_t key = order_key(r[t]);
+        uint8_t v = 0;
+        if (key > cut) v = 1;
+        else if (key == cut) { v = rank < remaining; ++rank; }
+        mask[t] = v;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// step 3: compaction.  Single pass: each CTA takes a tile of TILE tokens
+// (ticket order), ballots its mask, publishes the tile count, finds its output
+// base by decoupled look-back over the preceding tiles, then its warps move the
+// tile's active rows with 128-bit accesses.
+// ---------------------------------------------------------------------------
+struct RowStreams {
+    const char* src[DASH_MAX_ROW_STREAMS];
+    char* dst[DASH_MAX_ROW_STREAMS];
+    int64_t row_bytes[DASH_MAX_ROW_STREAMS], src_ld[DASH_MAX_ROW_STREAMS], dst_ld[DASH_MAX_ROW_STREAMS];
+    int vec16[DASH_MAX_ROW_STREAMS];
+    int count;
+};
+
+constexpr unsigned long long kFlagAgg = 1ull << 32, kFlagPrefix = 2ull << 32;
+
+__device__ __forceinline__ unsigned long long ld_state(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_state(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+template <int TILE>
+__global__ void __launch_bounds__(256)
+compact_kernel(const uint8_t* __restrict__ mask, int64_t n_upper, const int32_t* __restrict__ cu_in, int S,
+               RowStreams rs, const int32_t* __restrict__ pos_in, int32_t* __restrict__ pos_out,
+               const int32_t* __restrict__ tok_in, int32_t* __restrict__ tok_out,
+               int32_t* __restrict__ idx_out, int32_t* __restrict__ cu_out, int32_t* __restrict__ n_out_dev,
+               unsigned long long* tile_state, unsigned int* ticket, int* status) {
+    constexpr int NW = TILE / 32;                       // warps that ballot
+    __shared__ unsigned int s_ballot[NW];
+    __shared__ int s_wprefix[NW + 1];
+    __shared__ int s_src[TILE];
+    __shared__ int s_base;
+    __shared__ unsigned int s_tile;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
+    __syncthreads();
+    const int tile = (int)s_tile;
+    int64_t n = cu_in[S];
+    if (n > n_upper) n = n_upper;
+    const int64_t t_start = (int64_t)tile * TILE;
+    if (t_start >= n && tile != 0) return;              // nothing depends on tiles past the end
+    const int64_t t_end = (t_start + TILE < n) ? t_start + TILE : n;
+    const bool last_tile = (t_end >= n);
+
+    int my = 0;
+    if (warp < NW) {
+        int64_t t = t_start + threadIdx.x;
+        my = (t < n) ? (mask[t] != 0) : 0;
+        unsigned int bal = __ballot_sync(0xffffffffu, my);
+        if (lane == 0) s_ballot[warp] = bal;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int c = (lane < NW) ? __popc(s_ballot[lane]) : 0;
+        int inc = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int x = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += x;
+        }
+        if (lane < NW) s_wprefix[lane] = inc - c;
+        const int agg = __shfl_sync(0xffffffffu, inc, 31);
+        if (lane == 0) s_wprefix[NW] = agg;
+        // publish this tile's count, then look back
+        int base = 0;
+        if (tile == 0) {
+            if (lane == 0) st_state(&tile_state[0], kFlagPrefix | (unsigned int)agg);
+        } else {
+            if (lane == 0) st_state(&tile_state[tile], kFlagAgg | (unsigned int)agg);
+            int look = tile - 1;
+            bool done = false, timed_out = false;
+            while (!done) {
+                const int j = look - lane;
+                unsigned long long st = kFlagPrefix;    // virtual tiles before 0: prefix 0
+                uint32_t spins = 0;
+                if (j >= 0) {
+                    st = ld_state(&tile_state[j]);
+                    while ((st >> 32) == 0) {
+                        if (++spins > kSpinLimit) { timed_out = true; break; }
+                        __nanosleep(32);
+                        st = ld_state(&tile_state[j]);
+                    }
+                }
+                if (__any_sync(0xffffffffu, timed_out)) { timed_out = true; break; }
+                const unsigned int has_prefix = __ballot_sync(0xffffffffu, (st >> 32) == 2);
+                const int first = has_prefix ? (__ffs(has_prefix) - 1) : 32;   // nearest tile with a full prefix
+                int v = (lane <= first) ? (int)(unsigned int)(st & 0xffffffffu) : 0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                base += v;
+                if (has_prefix) done = true; else look -= 32;
+            }
+            if (timed_out) { if (lane == 0) atomicExch(status, DASH_ERR_TIMEOUT); base = 0; }
+            if (lane == 0) st_state(&tile_state[tile], kFlagPrefix | (unsigned int)(base + agg));
+        }
+        if (lane == 0) s_base = base;
+    }
+    __syncthreads();
+    const int base = s_base;
+    const int count = s_wprefix[NW];
+    if (warp < NW && my) {
+        int local = s_wprefix[warp] + __popc(s_ballot[warp] & ((1u << lane) - 1u));
+        int t = (int)(t_start + threadIdx.x);
+        s_src[local] = t;
+        if (idx_out) idx_out[base + local] = t;
+        if (pos_out) pos_out[base + local] = pos_in[t];
+        if (tok_out) tok_out[base + local] = tok_in[t];
+    }
+    // new sequence boundaries: cu_out[s] = number of active tokens before cu_in[s]
+    for (int s = threadIdx.x; s <= S; s += blockDim.x) {
+        int64_t c = cu_in[s];
+        if (c > n) c = n;
+        bool mine = (c >= t_start && c < t_start + TILE && c < t_end) || (last_tile && c == t_end);
+        if (tile == 0 && n == 0) mine = true;
+        if (mine) {
+            int p = (int)(c - t_start);
+            int v = base;
+            if (p >= TILE || c >= t_end) v += count;
+            else v += s_wprefix[p >> 5] + __popc(s_ballot[p >> 5] & ((1u << (p & 31)) - 1u));
+            cu_out[s] = v;
+            if (s == S && n_out_dev) *n_out_dev = v;
+        }
+    }
+    __syncthreads();
+    // move the rows
+    const int nwarps = blockDim.x >> 5;
+    for (int q = 0; q < rs.count; ++q) {
+        for (int k = warp; k < count; k += nwarps) {
+            const char* src = rs.src[q] + (int64_t)s_src[k] * rs.src_ld[q];
+            char* dst = rs.dst[q] + (int64_t)(base + k) * rs.dst_ld[q];
+            if (rs.vec16[q]) warp_copy_row16(src, dst, rs.row_bytes[q], lane);
+            else warp_copy_row4(src, dst, rs.row_bytes[q], lane);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+scatter_kernel(const char* __restrict__ src, int64_t n, int64_t row_bytes, int64_t src_ld, const int32_t* __restrict__ tok_index,
+               const uint8_t* __restrict__ sel, int which, const int32_t* __restrict__ n_dev, char* __restrict__ dst,
+               int64_t dst_ld, int vec16) {
+    const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+    if (n_dev) { int64_t nd = *n_dev; if (nd < n) n = nd; }
+    for (int64_t i = (int64_t)blockIdx.x * wpb + (threadIdx.x >> 5); i < n; i += (int64_t)gridDim.x * wpb) {
+        if (which != 2 && (int)(sel[i] != 0) != which) continue;
+        int64_t drow = tok_index ? (int64_t)tok_index[i] : i;
+        if (vec16) warp_copy_row16(src + i * src_ld, dst + drow * dst_ld, row_bytes, lane);
+        else warp_copy_row4(src + i * src_ld, dst + drow * dst_ld, row_bytes, lane);
+    }
+}
+
+static int rows_grid(int64_t n, int wpb) {
+    int64_t blocks = (n + wpb - 1) / wpb;
+    int64_t cap = (int64_t)sm_count() * 8;     // 8 CTAs of 256 threads fill an SM
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+}  // namespace dash
+
+using namespace dash;
+
+extern "C" int dash_delta_norm(const void* U, const void* H, int64_t n, int d, int64_t ldU, int64_t ldH,
+                               dash_dtype dt, dash_norm_mode mode, float eps, float* r_out,
+                               void* Hres_out, int64_t ldHres, const int32_t* res_index,
+                               const dash_threshold* fused, const int32_t* n_dev, void* stream) {
+    if (n < 0 || d <= 0 || (d % 8) != 0) return DASH_ERR_INVALID_ARG;
+    if (dt != DASH_F32 && dt != DASH_BF16) return DASH_ERR_INVALID_ARG;
+    if (mode != DASH_NORM_REL && mode != DASH_NORM_ABS) return DASH_ERR_INVALID_ARG;
+    if (n == 0) return DASH_OK;
+    const int es = (dt == DASH_BF16) ? 2 : 4;
+    const bool need_h = (mode == DASH_NORM_REL) || Hres_out;
+    if (!U || !r_out || (need_h && !H)) return DASH_ERR_INVALID_ARG;
+    if (ldU < d || (need_h && ldH < d) || (Hres_out && ldHres < d)) return DASH_ERR_INVALID_ARG;
+    if (!aligned16(U) || (need_h && !aligned16(H)) || (Hres_out && !aligned16(Hres_out))) return DASH_ERR_INVALID_ARG;
+    if ((ldU * es) % 16 || (need_h && (ldH * es) % 16) || (Hres_out && (ldHres * es) % 16)) return DASH_ERR_INVALID_ARG;
+    if (n > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
+    FusedThreshold ft = {0.f, 0, 0, nullptr, 0, nullptr};
+    if (fused) {
+        if (!fused->cu_seqlens || fused->S < 1 || !fused->mask_out || fused->keep_first < 0 || fused->keep_last < 0)
+            return DASH_ERR_INVALID_ARG;
+        ft = {fused->tau, fused->keep_first, fused->keep_last, fused->cu_seqlens, fused->S, fused->mask_out};
+    }
+    const int nvec = d * es / 16;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int grid = rows_grid(n, 8);
+    if (dt == DASH_BF16)
+        delta_norm_kernel<true><<<grid, 256, 0, st>>>((const char*)U, (const char*)H, n, nvec, ldU * es, ldH * es, (int)mode, eps,
+                                                      r_out, (char*)Hres_out, ldHres * es, res_index, ft, n_dev);
+    else
+        delta_norm_kernel<false><<<grid, 256, 0, st>>>((const char*)U, (const char*)H, n, nvec, ldU * es, ldH * es, (int)mode, eps,
+                                                       r_out, (char*)Hres_out, ldHres * es, res_index, ft, n_dev);
+    DASH_CUDA_TRY(cudaGetLastError());
+    return DASH_OK;
+}
+
+extern "C" int dash_select(const float* r, int64_t n, const int32_t* cu_seqlens, int S, dash_sel_mode mode, float tau,
+                           const int32_t* keep_counts, int keep_first, int keep_last, uint8_t* mask_out,
+                           void* ws, size_t ws_bytes, void* stream) {
+    (void)ws; (void)ws_bytes;
+    if (n < 0 || S < 1 || !cu_seqlens || keep_first < 0 || keep_last < 0) return DASH_ERR_INVALID_ARG;
+    if (mode != DASH_SEL_THRESHOLD && mode != DASH_SEL_KEEP_COUNT) return DASH_ERR_INVALID_ARG;
+    if (n > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
+    if (n == 0) return DASH_OK;
+    if (!r || !mask_out) return DASH_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (mode == DASH_SEL_THRESHOLD) {
+        int grid = (int)((n + 255) / 256);
+        int cap = sm_count() * 8;
+        if (grid > cap) grid = cap;
+        select_threshold_kernel<<<grid, 256, 0, st>>>(r, n, cu_seqlens, S, tau, keep_first, keep_last, mask_out);
+    } else {
+        if (!keep_counts) return DASH_ERR_INVALID_ARG;
+        select_keep_count_kernel<<<S, 1024, 0, st>>>(r, cu_seqlens, S, keep_counts, keep_first, keep_last, mask_out);
+    }
+    DASH_CUDA_TRY(cudaGetLastError());
+    return DASH_OK;
+}
+
+static int compact_tile_for(int64_t n) {
+    const int64_t want = 2LL * sm_count();
+    if (n / 256 >= want) return 256;
+    if (n / 128 >= want) return 128;
+    if (n / 64 >= want) return 64;
+    return 32;
+}
+
+static size_t compact_ws_bytes(int64_t n) {
+    int64_t tiles = (n + 31) / 32 + 1;
+    return align_up(256 + (size_t)tiles * 8, 256);
+}
+
+extern "C" int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
+                            const dash_rows* rows, int n_rows,
+                            const int32_t* pos_in, int32_t* pos_out, const int32_t* tok_in, int32_t* tok_out,
+                            int32_t* idx_out, int32_t* cu_out, int32_t* n_out_dev,
+                            void* ws, size_t ws_bytes, void* stream) {
+    if (n < 0 || S < 1 || !cu_in || !cu_out || n_rows < 0 || n_rows > DASH_MAX_ROW_STREAMS) return DASH_ERR_INVALID_ARG;
+    if (n > 0 && !mask) return DASH_ERR_INVALID_ARG;
+    if (n_rows > 0 && !rows) return DASH_ERR_INVALID_ARG;
+    if (n > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
+    if ((pos_out && !pos_in) || (tok_out && !tok_in)) return DASH_ERR_INVALID_ARG;
+    RowStreams rs;
+    rs.count = n_rows;
+    for (int q = 0; q < n_rows; ++q) {
+        const dash_rows& x = rows[q];
+        if (!x.src || !x.dst || x.row_bytes <= 0 || (x.row_bytes % 4) || x.src_ld_bytes < x.row_bytes || x.dst_ld_bytes < x.row_bytes)
+            return DASH_ERR_INVALID_ARG;
+        if ((x.src_ld_bytes % 4) || (x.dst_ld_bytes % 4) || ((uintptr_t)x.src % 4) || ((uintptr_t)x.dst % 4)) return DASH_ERR_INVALID_ARG;
+        rs.src[q] = (const char*)x.src; rs.dst[q] = (char*)x.dst;
+        rs.row_bytes[q] = x.row_bytes; rs.src_ld[q] = x.src_ld_bytes; rs.dst_ld[q] = x.dst_ld_bytes;
+        rs.vec16[q] = aligned16(x.src) && aligned16(x.dst) && !(x.row_bytes % 16) && !(x.src_ld_bytes % 16) && !(x.dst_ld_bytes % 16);
+    }
+    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < compact_ws_bytes(n)) return DASH_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int TILE = compact_tile_for(n);
+    const int tiles = (int)((n + TILE - 1) / TILE) > 0 ? (int)((n + TILE - 1) / TILE) : 1;
+    unsigned int* ticket = (unsigned int*)ws;
+    unsigned long long* state = (unsigned long long*)((char*)ws + 256);
+    DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)tiles * 8, st));
+    int* status = status_word_ptr();
+    if (!status) return DASH_ERR_CUDA;
+#define DASH_LAUNCH_COMPACT(T)                                                                                    \
+    compact_kernel<T><<<tiles, 256, 0, st>>>(mask, n, cu_in, S, rs, pos_in, pos_out, tok_in, tok_out, idx_out, \
+                                             cu_out, n_out_dev, state, ticket, status)
+    switch (TILE) {
+        case 256: DASH_LAUNCH_COMPACT(256); break;
+        case 128: DASH_LAUNCH_COMPACT(128); break;
+        case 64: DASH_LAUNCH_COMPACT(64); break;
+        default: DASH_LAUNCH_COMPACT(32); break;
+    }
+#undef DASH_LAUNCH_COMPACT
+    DASH_CUDA_TRY(cudaGetLastError());
+    return DASH_OK;
+}
+
+extern "C" int dash_scatter(const void* src, int64_t n, int64_t row_bytes, int64_t src_ld_bytes,
+                            const int32_t* tok_index, const uint8_t* sel, int which, const int32_t* n_dev,
+                            void* dst_full, int64_t dst_ld_bytes, void* stream) {
+    if (n < 0 || row_bytes <= 0 || (row_bytes % 4) || which < 0 || which > 2) return DASH_ERR_INVALID_ARG;
+    if (n == 0) return DASH_OK;
+    if (!src || !dst_full || (which != 2 && !sel)) return DASH_ERR_INVALID_ARG;
+    if (src_ld_bytes < row_bytes || dst_ld_bytes < row_bytes || (src_ld_bytes % 4) || (dst_ld_bytes % 4)) return DASH_ERR_INVALID_ARG;
+    if (((uintptr_t)src % 4) || ((uintptr_t)dst_full % 4)) return DASH_ERR_INVALID_ARG;
+    int vec16 = aligned16(src) && aligned16(dst_full) && !(row_bytes % 16) && !(src_ld_bytes % 16) && !(dst_ld_bytes % 16);
+    scatter_kernel<<<rows_grid(n, 8), 256, 0, (cudaStream_t)stream>>>((const char*)src, n, row_bytes, src_ld_bytes, tok_index, sel, which,
+                                                                       n_dev, (char*)dst_full, dst_ld_bytes, vec16);
+    DASH_CUDA_TRY(cudaGetLastError());
+    return DASH_OK;
+}
+
+namespace dash {
+size_t select_ws_bytes(int64_t, int) { return 256; }
+size_t compact_ws_bytes_pub(int64_t n) { return compact_ws_bytes(n); }
+}  // namespace dash

@@ -1,0 +1,285 @@
+"""Thin ctypes binding over the C-ABI CUDA library (include/dash.h).
+
+Argument marshalling only: every step of the path runs in the library's
+kernels.  Tensors are torch CUDA tensors (torch provides device memory and the
+current stream); nothing here computes on the host.  If the library cannot be
+loaded the import of a symbol raises -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import (POINTER, Structure, c_char_p, c_double, c_float, c_int, c_int32, c_int64,
+                    c_size_t, c_uint8, c_void_p)
+from typing import Optional, Sequence
+
+import torch
+
+F32, BF16 = 0, 1
+NORM_REL, NORM_ABS = 0, 1
+SEL_THRESHOLD, SEL_KEEP_COUNT = 0, 1
+WS_SELECT, WS_COMPACT, WS_ATTENTION = 0, 1, 2
+OK = 0
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdash.so")
+
+EXPORTS = [
+    "dash_status_string", "dash_check_status", "dash_keep_count", "dash_flops_per_layer", "dash_flops_speedup",
+    "dash_delta_norm", "dash_select", "dash_compact", "dash_scatter", "dash_varlen_attention",
+    "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes",
+]
+
+
+class Threshold(Structure):
+    _fields_ = [("tau", c_float), ("keep_first", c_int), ("keep_last", c_int),
+                ("cu_seqlens", c_void_p), ("S", c_int), ("mask_out", c_void_p)]
+
+
+class Rows(Structure):
+    _fields_ = [("src", c_void_p), ("dst", c_void_p), ("row_bytes", c_int64),
+                ("src_ld_bytes", c_int64), ("dst_ld_bytes", c_int64)]
+
+
+class LayerCfg(Structure):
+    _fields_ = [("d", c_int), ("Hq", c_int), ("Hkv", c_int), ("D", c_int), ("dt", c_int),
+                ("Wqkv", c_void_p), ("Wo", c_void_p), ("rms_weight", c_void_p), ("rms_eps", c_float),
+                ("rope_base", c_double), ("norm_mode", c_int), ("norm_eps", c_float), ("sel_mode", c_int),
+                ("tau", c_float), ("keep_counts", c_void_p), ("keep_first", c_int), ("keep_last", c_int),
+                ("scatter_which", c_int)]
+
+
+class LayerWsLayout(Structure):
+    _fields_ = [("Hn", c_size_t), ("QKV", c_size_t), ("O", c_size_t), ("U", c_size_t), ("Ht", c_size_t),
+                ("scratch", c_size_t), ("total", c_size_t)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libdash.so (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2604_18103_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.dash_status_string.restype = c_char_p
+        L.dash_status_string.argtypes = [c_int]
+        L.dash_check_status.argtypes = [c_void_p]
+        L.dash_keep_count.restype = c_int64
+        L.dash_keep_count.argtypes = [c_int64, c_double, c_int, c_int, c_int]
+        L.dash_flops_per_layer.restype = c_double
+        L.dash_flops_per_layer.argtypes = [c_double] * 3
+        L.dash_flops_speedup.restype = c_double
+        L.dash_flops_speedup.argtypes = [c_double, c_double, c_int, c_int, c_double, c_double]
+        L.dash_delta_norm.argtypes = [c_void_p, c_void_p, c_int64, c_int, c_int64, c_int64, c_int, c_int, c_float,
+                                      c_void_p, c_void_p, c_int64, c_void_p, POINTER(Threshold), c_void_p, c_void_p]
+        L.dash_select.argtypes = [c_void_p, c_int64, c_void_p, c_int, c_int, c_float, c_void_p, c_int, c_int,
+                                  c_void_p, c_void_p, c_size_t, c_void_p]
+        L.dash_compact.argtypes = [c_void_p, c_int64, c_void_p, c_int, POINTER(Rows), c_int, c_void_p, c_void_p,
+                                   c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.dash_scatter.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_int, c_void_p,
+                                   c_void_p, c_int64, c_void_p]
+        L.dash_varlen_attention.argtypes = [c_void_p] * 5 + [c_int64] * 4 + [c_void_p, c_int, c_int64, c_int64,
+                                                                          c_int, c_int, c_int, c_float, c_int, c_int,
+                                                                          c_void_p, c_size_t, c_void_p]
+        L.dash_layer_workspace.argtypes = [POINTER(LayerCfg), c_int64, c_int, POINTER(LayerWsLayout)]
+        L.dash_layer_step.argtypes = [POINTER(LayerCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
+                                      c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                      c_void_p, c_size_t, c_void_p]
+        L.dash_workspace_bytes.restype = c_size_t
+        L.dash_workspace_bytes.argtypes = [c_int, c_int64, c_int, c_int, c_int, c_int, c_int]
+        _lib = L
+    return _lib
+
+
+class DashError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib().dash_status_string(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise DashError(status, where)
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream():
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _dev(t: torch.Tensor, *more):
+    for x in (t, *more):
+        if x is not None and not x.is_cuda:
+            raise ValueError("device tensor expected")
+
+
+# ---- host helpers -------------------------------------------------------------
+def dash_keep_count(n: int, rho: float, keep_first: int = 0, keep_last: int = 0, mode: int = 0) -> int:
+    return int(lib().dash_keep_count(n, rho, keep_first, keep_last, mode))
+
+
+def dash_flops_per_layer(n, d, m) -> float:
+    return float(lib().dash_flops_per_layer(n, d, m))
+
+
+def dash_flops_speedup(n, n_hat, L, l_s, d, m) -> float:
+    return float(lib().dash_flops_speedup(n, n_hat, L, l_s, d, m))
+
+
+def dash_check_status() -> int:
+    return int(lib().dash_check_status(_stream()))
+
+
+def dash_workspace_bytes(op: int, n: int, S: int = 1, Hq: int = 0, Hkv: int = 0, D: int = 0, dt: int = BF16) -> int:
+    return int(lib().dash_workspace_bytes(op, n, S, Hq, Hkv, D, dt))
+
+
+def workspace(nbytes: int, device) -> torch.Tensor:
+    """256-byte aligned scratch buffer (torch's caching allocator aligns to 512)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+# ---- step 1 ---------------------------------------------------------------------
+def dash_delta_norm(U: torch.Tensor, H: Optional[torch.Tensor], mode: int = NORM_REL, eps: float = 1e-12,
+                    r_out: Optional[torch.Tensor] = None, Hres_out: Optional[torch.Tensor] = None,
+                    res_index: Optional[torch.Tensor] = None, tau: Optional[float] = None,
+                    cu_seqlens: Optional[torch.Tensor] = None, keep_first: int = 0, keep_last: int = 0,
+                    mask_out: Optional[torch.Tensor] = None, n_dev: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _dev(U, H, r_out, Hres_out)
+    n, d = U.shape
+    if r_out is None:
+        r_out = torch.empty(n, dtype=torch.float32, device=U.device)
+    fused = None
+    if mask_out is not None:
+        fused = Threshold(float(tau), keep_first, keep_last, cu_seqlens.data_ptr(), cu_seqlens.numel() - 1, mask_out.data_ptr())
+    st = lib().dash_delta_norm(_p(U), _p(H), n, d, U.stride(0), H.stride(0) if H is not None else d, dtype_code(U), mode, eps,
+                               _p(r_out), _p(Hres_out), Hres_out.stride(0) if Hres_out is not None else d, _p(res_index),
+                               ctypes.byref(fused) if fused is not None else None, _p(n_dev), _stream())
+    _check(st, "dash_delta_norm")
+    return r_out
+
+
+# ---- step 2 ---------------------------------------------------------------------
+def dash_select(r: torch.Tensor, cu_seqlens: torch.Tensor, mode: int, tau: float = 0.0,
+                keep_counts: Optional[torch.Tensor] = None, keep_first: int = 0, keep_last: int = 0,
+                mask_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _dev(r, cu_seqlens, keep_counts)
+    n = r.numel()
+    if mask_out is None:
+        mask_out = torch.empty(n, dtype=torch.uint8, device=r.device)
+    st = lib().dash_select(_p(r), n, _p(cu_seqlens), cu_seqlens.numel() - 1, mode, tau, _p(keep_counts), keep_first, keep_last,
+                           _p(mask_out), None, 0, _stream())
+    _check(st, "dash_select")
+    return mask_out
+
+
+# ---- step 3 ---------------------------------------------------------------------
+def dash_compact(mask: torch.Tensor, cu_in: torch.Tensor, rows: Sequence[torch.Tensor] = (),
+                 rows_out: Optional[Sequence[torch.Tensor]] = None, pos_in: Optional[torch.Tensor] = None,
+                 tok_in: Optional[torch.Tensor] = None, want_idx: bool = True, ws: Optional[torch.Tensor] = None):
+    """Returns dict(idx, cu_out, n_out (device int32 [1]), rows (list), pos_out, tok_out); outputs are sized n."""
+    _dev(mask, cu_in)
+    n = mask.numel()
+    S = cu_in.numel() - 1
+    dev = mask.device
+    if rows_out is None:
+        rows_out = [torch.empty_like(x) for x in rows]
+    arr = (Rows * max(len(rows), 1))()
+    for i, (x, y) in enumerate(zip(rows, rows_out)):
+        rb = x.shape[1] * x.element_size() if x.dim() > 1 else x.element_size()
+        rb = int(x[0].numel() * x.element_size()) if x.shape[0] > 0 else rb
+        arr[i] = Rows(x.data_ptr(), y.data_ptr(), rb, x.stride(0) * x.element_size(), y.stride(0) * y.element_size())
+    idx = torch.empty(n, dtype=torch.int32, device=dev) if want_idx else None
+    pos_out = torch.empty(n, dtype=torch.int32, device=dev) if pos_in is not None else None
+    tok_out = torch.empty(n, dtype=torch.int32, device=dev) if tok_in is not None else None
+    cu_out = torch.empty(S + 1, dtype=torch.int32, device=dev)
+    n_out = torch.empty(1, dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = workspace(dash_workspace_bytes(WS_COMPACT, n, S), dev)
+    st = lib().dash_compact(_p(mask), n, _p(cu_in), S, arr, len(rows), _p(pos_in), _p(pos_out), _p(tok_in), _p(tok_out),
+                            _p(idx), _p(cu_out), _p(n_out), _p(ws), ws.numel(), _stream())
+    _check(st, "dash_compact")
+    return {"idx": idx, "cu_out": cu_out, "n_out": n_out, "rows": list(rows_out), "pos_out": pos_out, "tok_out": tok_out}
+
+
+def dash_scatter(src: torch.Tensor, dst_full: torch.Tensor, tok_index: Optional[torch.Tensor] = None,
+                 sel: Optional[torch.Tensor] = None, which: int = 2, n_dev: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _dev(src, dst_full, tok_index, sel)
+    n = src.shape[0]
+    rb = int(src[0].numel() * src.element_size()) if n > 0 else 4
+    st = lib().dash_scatter(_p(src), n, rb, src.stride(0) * src.element_size(), _p(tok_index), _p(sel), which, _p(n_dev),
+                            _p(dst_full), dst_full.stride(0) * dst_full.element_size(), _stream())
+    _check(st, "dash_scatter")
+    return dst_full
+
+
+# ---- step 4 ---------------------------------------------------------------------
+def dash_varlen_attention(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, cu_seqlens: torch.Tensor, max_seqlen: int,
+                          scale: Optional[float] = None, O: Optional[torch.Tensor] = None, want_lse: bool = False,
+                          ws: Optional[torch.Tensor] = None):
+    """Q [n,Hq,D], K,V [n,Hkv,D] (last two dims contiguous).  Returns O (and lse [Hq,n] if asked)."""
+    _dev(Q, K, V, cu_seqlens)
+    n, Hq, D = Q.shape
+    Hkv = K.shape[1]
+    if scale is None:
+        scale = 1.0 / (D ** 0.5)
+    if O is None:
+        O = torch.empty(n, Hq, D, dtype=Q.dtype, device=Q.device)
+    lse = torch.empty(Hq, n, dtype=torch.float32, device=Q.device) if want_lse else None
+    dt = dtype_code(Q)
+    if ws is None:
+        ws = workspace(dash_workspace_bytes(WS_ATTENTION, n, cu_seqlens.numel() - 1, Hq, Hkv, D, dt), Q.device)
+    st = lib().dash_varlen_attention(_p(Q), _p(K), _p(V), _p(O), _p(lse), Q.stride(0), K.stride(0), V.stride(0), O.stride(0),
+                                     _p(cu_seqlens), cu_seqlens.numel() - 1, n, int(max_seqlen), Hq, Hkv, D, float(scale), 1, dt,
+                                     _p(ws), ws.numel(), _stream())
+    _check(st, "dash_varlen_attention")
+    return (O, lse) if want_lse else O
+
+
+# ---- the block step ---------------------------------------------------------------
+class Layer:
+    """Device-resident weights and configuration of one block for dash_layer_step."""
+
+    def __init__(self, shape, weights, device, norm_mode=NORM_REL, norm_eps=1e-12, sel_mode=SEL_THRESHOLD, tau=0.0,
+                 keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2):
+        self.shape = shape
+        self.Wqkv = torch.cat([weights["Wq"], weights["Wk"], weights["Wv"]], dim=1).contiguous().to(device)
+        self.Wo = weights["Wo"].contiguous().to(device)
+        self.rms_w = weights["rms_w"].contiguous().to(device)
+        self.keep_counts = keep_counts
+        self.cfg = LayerCfg(shape.d, shape.Hq, shape.Hkv, shape.D, dtype_code(self.Wo), self.Wqkv.data_ptr(), self.Wo.data_ptr(),
+                            self.rms_w.data_ptr(), shape.rms_eps, shape.rope_base, norm_mode, norm_eps, sel_mode, tau,
+                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which)
+
+    def set_tau(self, tau: float):
+        self.cfg.tau = float(tau)
+
+
+def dash_layer_workspace(layer: Layer, n: int, S: int) -> LayerWsLayout:
+    out = LayerWsLayout()
+    _check(lib().dash_layer_workspace(ctypes.byref(layer.cfg), n, S, ctypes.byref(out)), "dash_layer_workspace")
+    return out
+
+
+def dash_layer_step(layer: Layer, H_in, tok_index_in, pos_in, cu_in, max_seqlen: int, x_full, H_next, tok_index_next, pos_next,
+                    cu_next, n_next, r_out, mask_out, ws):
+    n = H_in.shape[0]
+    st = lib().dash_layer_step(ctypes.byref(layer.cfg), _p(H_in), _p(tok_index_in), _p(pos_in), _p(cu_in), cu_in.numel() - 1, n,
+                               int(max_seqlen), _p(x_full), _p(H_next), _p(tok_index_next), _p(pos_next), _p(cu_next), _p(n_next),
+                               _p(r_out), _p(mask_out), _p(ws), ws.numel(), _stream())
+    _check(st, "dash_layer_step")
