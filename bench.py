@@ -68,7 +68,7 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
 
-    def stop(self):
+    def stop(self, first: int = 0):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -77,7 +77,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        for r in self.rows:
+        for r in self.rows[max(0, first - 1):]:
             try:
                 sm.append(float(r[1])); mx.append(float(r[2]))
             except Exception:
@@ -143,6 +143,7 @@ def run_ours(args):
     r = torch.zeros(T, dtype=torch.float32, device=dev)
     mask = torch.zeros(T, dtype=torch.uint8, device=dev)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush_src = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device=dev)
     # host-side result buffers of the end-to-end arm
     x_full_h = torch.empty(T, sh.d, dtype=sh.dtype).pin_memory()
     H_next_h = torch.empty(T, sh.d, dtype=sh.dtype).pin_memory()
@@ -163,6 +164,9 @@ def run_ours(args):
     def step():
         dash.dash_layer_step(layer, H, tok, pos, cu, T, x_full, H_next, tok_next, pos_next, cu_next, n_next, r, mask, ws)
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     h2d()
     # threshold at the 40th percentile of the measured relative delta (harness work, untimed)
     step()
@@ -185,7 +189,8 @@ def run_ours(args):
         evs = []
         barrier()
         for _ in range(steps):
-            flush.zero_()
+            flush.zero_()          # write a buffer larger than L2 ...
+            flush_src.sum()        # ... then read another one, so the timed kernels do not inherit dirty-line write-backs
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             if pre:
@@ -198,12 +203,14 @@ def run_ours(args):
         barrier()
         return [a.elapsed_time(b) for a, b in evs]
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    if rank == 0:                                   # the sampler needs a moment before its first line
+        t_s = time.time()
+        while not sampler.rows and time.time() - t_s < 5.0:
+            step()
+            torch.cuda.synchronize()
+    n_before = len(sampler.rows)
     t_wall0 = time.time()
     ms = timed(step, args.steps)
-    clocks = sampler.stop() if rank == 0 else None
     wall = time.time() - t_wall0
     ms_e2e = timed(step, max(3, min(args.steps, 10)), pre=h2d, post=d2h)
 
@@ -224,6 +231,7 @@ def run_ours(args):
     cws = dash.workspace(dash.dash_workspace_bytes(dash.WS_COMPACT, T, S), dev)
     ms_comp = timed(lambda: dash.dash_compact(mask, cu, rows=[Ht], rows_out=[H_next], pos_in=pos, tok_in=tok, want_idx=False, ws=cws), 10)
     status = dash.dash_check_status()
+    clocks = sampler.stop(n_before) if rank == 0 else None
 
     def reduce_max(x):
         if world == 1:
@@ -253,7 +261,7 @@ def run_ours(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"configs[1]: Qwen2.5-7B-shaped single layer, bf16, batch 1, seq {T}, threshold at 40th percentile "
                                f"({n_active} of {T} tokens stay active)", "tokens_per_step_per_gpu": T, "n_active_after": n_active,
-                   "tau": tau, "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write)",
+                   "tau": tau, "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write, then {L2_FLUSH_BYTES >> 20} MiB read)",
                    "status_word": status},
         "e2e": {"value": world * T / (t_e2e * 1e-3), "unit": UNIT, "ms_per_step": t_e2e, "h2d_bytes_per_step": h2d_bytes,
                 "d2h_bytes_per_step": d2h_bytes},
@@ -356,7 +364,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--seq", type=int, default=8192)

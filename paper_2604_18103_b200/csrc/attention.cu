@@ -65,6 +65,11 @@ constexpr int kBN = 128;                 // keys per block
 constexpr int kAttnThreads = 160;
 constexpr long long kWaitCycles = 4000000000LL;   // ~2 s: a wait that long is reported, not retried
 constexpr uint32_t kTmemCols = 256;
+// how many of every four exponentials are evaluated on the FMA pipe instead of the MUFU
+#ifndef DASH_EXP_POLY_PER4
+#define DASH_EXP_POLY_PER4 1
+#endif
+constexpr int kExpPolyPer4 = DASH_EXP_POLY_PER4;
 
 struct AttnParams {
     const int32_t* cu;
@@ -200,32 +205,46 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_base + c * 32, &sreg[c * 32]);
             tmem_wait_ld();
             const bool diag = (j == qt);
-            float mx = -INFINITY;
+            if (diag) {
 #pragma unroll
-            for (int c = 0; c < 128; ++c) {
-                float v = __uint_as_float(sreg[c]);
-                if (diag && c > row) v = -INFINITY;
-                sreg[c] = __float_as_uint(v);
-                mx = fmaxf(mx, v);
+                for (int c = 0; c < 128; ++c)
+                    if (c > row) sreg[c] = 0xff800000u;     // -inf: keys after the query (and past the sequence end)
             }
-            const float m_new = fmaxf(m, mx);
+            // four independent chains keep the max / sum reductions off the latency-bound path
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 128; c += 4) {
+                mx0 = fmaxf(mx0, __uint_as_float(sreg[c]));     mx1 = fmaxf(mx1, __uint_as_float(sreg[c + 1]));
+                mx2 = fmaxf(mx2, __uint_as_float(sreg[c + 2])); mx3 = fmaxf(mx3, __uint_as_float(sreg[c + 3]));
+            }
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+            // Lazy rescale: the reference max m only moves when the block max exceeds it by more than
+            // 2^8 in the exponent; until then P is formed against the old m (values up to 256, safe in
+            // bf16 / fp32) and O needs no correction.
+            const bool grow = (mx - m) * p.scale_log2 > 8.0f;
+            const float m_new = grow ? mx : m;
             const float msl = m_new * p.scale_log2;
-            const float alpha = ex2((m - m_new) * p.scale_log2);
-            float sum = 0.f;
+            const float alpha = grow ? ex2((m - m_new) * p.scale_log2) : 1.0f;
+            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-            for (int c = 0; c < 128; c += 2) {
+            for (int c = 0; c < 128; c += 4) {
                 float p0 = ex2(fmaf(__uint_as_float(sreg[c]), p.scale_log2, -msl));
-                float p1 = ex2(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl));
-                sum += p0 + p1;
+                float p1 = (kExpPolyPer4 >= 2) ? ex2_poly(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl))
+                                               : ex2(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl));
+                float p2 = ex2(fmaf(__uint_as_float(sreg[c + 2]), p.scale_log2, -msl));
+                float p3 = (kExpPolyPer4 >= 1) ? ex2_poly(fmaf(__uint_as_float(sreg[c + 3]), p.scale_log2, -msl))
+                                               : ex2(fmaf(__uint_as_float(sreg[c + 3]), p.scale_log2, -msl));
+                sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
                 sreg[c >> 1] = pack_bf16(p0, p1);
+                sreg[(c >> 1) + 1] = pack_bf16(p2, p3);
             }
-            l = l * alpha + sum;
+            l = l * alpha + ((sum0 + sum1) + (sum2 + sum3));
             m = m_new;
             tmem_st32(tP + lane_base, &sreg[0]);
             tmem_st32(tP + lane_base + 32, &sreg[32]);
             if (j > 0) {
                 // O still holds the previous blocks' sum scaled by the old max
-                const bool need = __any_sync(0xffffffffu, alpha != 1.0f);
+                const bool need = __any_sync(0xffffffffu, grow);
                 if (need) {
                     ok = mbar_wait(bar_o, (j - 1) & 1, kWaitCycles);
                     if (!ok) break;

@@ -57,15 +57,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Copy one row of `bytes` (multiple of 16, 16-byte aligned ends) with a warp.
 __device__ __forceinline__ void warp_copy_row16(const char* __restrict__ src, char* __restrict__ dst, int64_t bytes, int lane) {
     const int nvec = (int)(bytes >> 4);
-    for (int base = 0; base < nvec; base += 32 * 4) {
-        uint4 r[4];
+    constexpr int UN = 8;                       // 8 x 16 B per lane in flight: 4 KB per warp
+    for (int base = 0; base < nvec; base += 32 * UN) {
+        uint4 r[UN];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < UN; ++k) {
             int v = base + k * 32 + lane;
             if (v < nvec) r[k] = ld_nc_v4(src + ((int64_t)v << 4));
         }
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < UN; ++k) {
             int v = base + k * 32 + lane;
             if (v < nvec) st_v4(dst + ((int64_t)v << 4), r[k]);
         }
