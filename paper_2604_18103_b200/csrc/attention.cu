@@ -101,7 +101,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base + L::kQ, sK = smem_base + L::kK, sV = smem_base + L::kV;
     const uint32_t bars = smem_base + L::kBars;
-    const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_o = bars + 32, bar_p = bars + 40;
+    const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_o = bars + 32, bar_p0 = bars + 40, bar_p1 = bars + 48;
     const uint32_t tmem_slot = bars + 64;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 64);
@@ -124,7 +124,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     if (warp == 4) {
         if (lane == 0) {
             mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1);
-            mbar_init(bar_s, 1); mbar_init(bar_o, 1); mbar_init(bar_p, 128);
+            mbar_init(bar_s, 1); mbar_init(bar_o, 1); mbar_init(bar_p0, 128); mbar_init(bar_p1, 128);
             *abort_gen = 0;
             fence_barrier_init();
             fence_proxy_async_smem();
@@ -152,11 +152,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, kvh, seq_a);
             mbar_arrive_expect_tx(bar_v, L::kTileBytes);
             for (int c = 0; c < KCH; ++c) tma_load_3d(sV + c * kChunkBytes, &mapV, bar_v, c * 64, kvh, seq_a);
-            ok = mbar_wait(bar_q, 0, kWaitCycles);
-            for (int j = 0; j < nblk && ok; ++j) {
-                const uint32_t ph = j & 1;
-                ok = ok && mbar_wait(bar_k, ph, kWaitCycles);
-                if (!ok) break;
+            auto issue_s = [&]() {
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
@@ -164,21 +160,40 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), idesc_s, kk > 0);
                 }
                 tc_commit(bar_s);
+            };
+            ok = mbar_wait(bar_q, 0, kWaitCycles) && mbar_wait(bar_k, 0, kWaitCycles);
+            if (ok) issue_s();
+            for (int j = 0; j < nblk && ok; ++j) {
+                const uint32_t ph = j & 1;
+                // S_j done: the K buffer is free for the next block
                 ok = mbar_wait(bar_s, ph, kWaitCycles);
                 if (!ok) break;
                 if (j + 1 < nblk) {
                     mbar_arrive_expect_tx(bar_k, L::kTileBytes);
                     for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, kvh, seq_a + (j + 1) * kBN);
                 }
-                ok = mbar_wait(bar_p, ph, kWaitCycles) && mbar_wait(bar_v, ph, kWaitCycles);
+                // O += P_j V_j, started as soon as the first 64 keys of P are in TMEM
+                ok = mbar_wait(bar_p0, ph, kWaitCycles) && mbar_wait(bar_v, ph, kWaitCycles);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < kBN / 16; ++kk) {
-                    // P: 128 lanes x (16 keys = 8 packed columns) per step; V: 16 keys = two 8-row groups of 1 KB
+                for (int kk = 0; kk < kBN / 32; ++kk)
                     mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
-                }
+                ok = mbar_wait(bar_p1, ph, kWaitCycles);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = kBN / 32; kk < kBN / 16; ++kk)
+                    mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, 1);
                 tc_commit(bar_o);
+                // S_{j+1} goes into the pipe right behind PV_j: tcgen05.mma of one thread execute in issue
+                // order, so PV_j has read P_j before S_{j+1} overwrites the columns they share
+                if (j + 1 < nblk) {
+                    ok = mbar_wait(bar_k, (j + 1) & 1, kWaitCycles);
+                    if (!ok) break;
+                    issue_s();
+                }
+                // PV_j done: the V buffer is free
                 ok = mbar_wait(bar_o, ph, kWaitCycles);
                 if (!ok) break;
                 if (j + 1 < nblk) {
@@ -225,38 +240,23 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             const float m_new = grow ? mx : m;
             const float msl = m_new * p.scale_log2;
             const float alpha = grow ? ex2((m - m_new) * p.scale_log2) : 1.0f;
-            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-#pragma unroll
-            for (int c = 0; c < 128; c += 4) {
-                float p0 = ex2(fmaf(__uint_as_float(sreg[c]), p.scale_log2, -msl));
-                float p1 = (kExpPolyPer4 >= 2) ? ex2_poly(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl))
-                                               : ex2(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl));
-                float p2 = ex2(fmaf(__uint_as_float(sreg[c + 2]), p.scale_log2, -msl));
-                float p3 = (kExpPolyPer4 >= 1) ? ex2_poly(fmaf(__uint_as_float(sreg[c + 3]), p.scale_log2, -msl))
-                                               : ex2(fmaf(__uint_as_float(sreg[c + 3]), p.scale_log2, -msl));
-                sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
-                sreg[c >> 1] = pack_bf16(p0, p1);
-                sreg[(c >> 1) + 1] = pack_bf16(p2, p3);
-            }
-            l = l * alpha + ((sum0 + sum1) + (sum2 + sum3));
-            m = m_new;
-            tmem_st32(tP + lane_base, &sreg[0]);
-            tmem_st32(tP + lane_base + 32, &sreg[32]);
             if (j > 0) {
-                // O still holds the previous blocks' sum scaled by the old max
+                // O still holds the previous blocks' sum scaled by the old reference max
                 const bool need = __any_sync(0xffffffffu, grow);
                 if (need) {
                     ok = mbar_wait(bar_o, (j - 1) & 1, kWaitCycles);
                     if (!ok) break;
                     tc_fence_after();
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(tO + lane_base + c * 32, o);
+                    // rare path (the reference max moves in the first blocks only): small chunks, not
+                    // unrolled, so it adds no register pressure to the hot loop around it
+#pragma unroll 1
+                    for (int c = 0; c < D / 8; ++c) {
+                        uint32_t o[8];
+                        tmem_ld8(tO + lane_base + c * 8, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        tmem_st32(tO + lane_base + c * 32, o);
+                        for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tmem_st8(tO + lane_base + c * 8, o);
                     }
                 }
             }
@@ -275,9 +275,29 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     fence_proxy_async_smem();
                 }
             }
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar_p);
+            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                for (int c = half * 64; c < half * 64 + 64; c += 4) {
+                    float p0 = ex2(fmaf(__uint_as_float(sreg[c]), p.scale_log2, -msl));
+                    float p1 = (kExpPolyPer4 >= 2) ? ex2_poly(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl))
+                                                   : ex2(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl));
+                    float p2 = ex2(fmaf(__uint_as_float(sreg[c + 2]), p.scale_log2, -msl));
+                    float p3 = (kExpPolyPer4 >= 1) ? ex2_poly(fmaf(__uint_as_float(sreg[c + 3]), p.scale_log2, -msl))
+                                                   : ex2(fmaf(__uint_as_float(sreg[c + 3]), p.scale_log2, -msl));
+                    sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+                    sreg[c >> 1] = pack_bf16(p0, p1);
+                    sreg[(c >> 1) + 1] = pack_bf16(p2, p3);
+                }
+                // the first 64 keys of P go out (and their PV steps start) while the rest is still being formed
+                tmem_st32(tP + lane_base + half * 32, &sreg[half * 32]);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(half == 0 ? bar_p0 : bar_p1);
+            }
+            l = l * alpha + ((sum0 + sum1) + (sum2 + sum3));
+            m = m_new;
         }
         if (ok) ok = mbar_wait(bar_o, (nblk - 1) & 1, kWaitCycles);
         if (ok && !*abort_gen) {
