@@ -67,7 +67,7 @@ constexpr long long kWaitCycles = 4000000000LL;   // ~2 s: a wait that long is r
 constexpr uint32_t kTmemCols = 256;
 // how many of every four exponentials are evaluated on the FMA pipe instead of the MUFU
 #ifndef DASH_EXP_POLY_PER4
-#define DASH_EXP_POLY_PER4 1
+#define DASH_EXP_POLY_PER4 0
 #endif
 constexpr int kExpPolyPer4 = DASH_EXP_POLY_PER4;
 
@@ -225,12 +225,14 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 for (int c = 0; c < 128; ++c)
                     if (c > row) sreg[c] = 0xff800000u;     // -inf: keys after the query (and past the sequence end)
             }
-            // four independent chains keep the max / sum reductions off the latency-bound path
+            // four independent chains of three-input max keep the reduction short and off the latency-bound path
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 128; c += 4) {
-                mx0 = fmaxf(mx0, __uint_as_float(sreg[c]));     mx1 = fmaxf(mx1, __uint_as_float(sreg[c + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(sreg[c + 2])); mx3 = fmaxf(mx3, __uint_as_float(sreg[c + 3]));
+            for (int c = 0; c < 128; c += 8) {
+                mx0 = fmax3(mx0, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
+                mx1 = fmax3(mx1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+                mx2 = fmax3(mx2, __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
+                mx3 = fmax3(mx3, __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
             }
             const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             // Lazy rescale: the reference max m only moves when the block max exceeds it by more than
@@ -275,20 +277,24 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     fence_proxy_async_smem();
                 }
             }
-            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+            // scale-subtract and row sums on packed fp32 pairs (two lanes per FMA-pipe instruction)
+            float2 sumA = make_float2(0.f, 0.f), sumB = make_float2(0.f, 0.f);
+            const float2 sl2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-msl, -msl);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
 #pragma unroll
                 for (int c = half * 64; c < half * 64 + 64; c += 4) {
-                    float p0 = ex2(fmaf(__uint_as_float(sreg[c]), p.scale_log2, -msl));
-                    float p1 = (kExpPolyPer4 >= 2) ? ex2_poly(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl))
-                                                   : ex2(fmaf(__uint_as_float(sreg[c + 1]), p.scale_log2, -msl));
-                    float p2 = ex2(fmaf(__uint_as_float(sreg[c + 2]), p.scale_log2, -msl));
-                    float p3 = (kExpPolyPer4 >= 1) ? ex2_poly(fmaf(__uint_as_float(sreg[c + 3]), p.scale_log2, -msl))
-                                                   : ex2(fmaf(__uint_as_float(sreg[c + 3]), p.scale_log2, -msl));
-                    sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
-                    sreg[c >> 1] = pack_bf16(p0, p1);
-                    sreg[(c >> 1) + 1] = pack_bf16(p2, p3);
+                    const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), sl2, nm2);
+                    const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), sl2, nm2);
+                    float2 pa, pb;
+                    pa.x = ex2(xa.x);
+                    pa.y = (kExpPolyPer4 >= 2) ? ex2_poly(xa.y) : ex2(xa.y);
+                    pb.x = ex2(xb.x);
+                    pb.y = (kExpPolyPer4 >= 1) ? ex2_poly(xb.y) : ex2(xb.y);
+                    sumA = __fadd2_rn(sumA, pa);
+                    sumB = __fadd2_rn(sumB, pb);
+                    sreg[c >> 1] = pack_bf16(pa.x, pa.y);
+                    sreg[(c >> 1) + 1] = pack_bf16(pb.x, pb.y);
                 }
                 // the first 64 keys of P go out (and their PV steps start) while the rest is still being formed
                 tmem_st32(tP + lane_base + half * 32, &sreg[half * 32]);
@@ -296,7 +302,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 tc_fence_before();
                 mbar_arrive(half == 0 ? bar_p0 : bar_p1);
             }
-            l = l * alpha + ((sum0 + sum1) + (sum2 + sum3));
+            l = l * alpha + ((sumA.x + sumA.y) + (sumB.x + sumB.y));
             m = m_new;
         }
         if (ok) ok = mbar_wait(bar_o, (nblk - 1) & 1, kWaitCycles);

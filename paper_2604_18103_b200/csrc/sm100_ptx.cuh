@@ -171,6 +171,13 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
+// three-input maximum (one instruction on sm_100)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // 2^x on the FMA pipe (no MUFU), for x <= 2^21: split x = floor(x) + f with a round-down add of
 // 1.5 * 2^23 (the integer lands in the low mantissa bits), evaluate a cubic fit of 2^f on [0,1)
 // (max relative error 8.7e-5, far below the bf16 rounding applied to P afterwards) and add
