@@ -51,9 +51,15 @@ def test_config2_block_step_full_size():
     torch.cuda.synchronize()
     assert dash.dash_check_status() == dash.OK
     O = bufs.view(bufs.lay.O, T, sh.Hq * sh.D, sh.dtype)[rows].float().cpu().numpy()
-    # O is an intermediate of the step: it inherits the bf16 rounding of the stored Q, K, V (twice the bar, as for those)
-    assert_close_rms(O.reshape(len(rows), sh.Hq, sh.D), ref["O"], "attention O (sampled rows)", tol=4e-2)
-    assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype)[rows].float().cpu().numpy(), ref["U"], "U (sampled rows)")
+    # O is an intermediate of the step: it inherits the rounding of the stored V (an early token may copy one value
+    # row almost unchanged), i.e. up to half a bf16 ulp of the largest |v| on top of the bar
+    half_ulp_v = 2.0 ** (math.floor(math.log2(float(np.abs(ref["V"]).max()))) - 8)
+    assert_close_rms(O.reshape(len(rows), sh.Hq, sh.D), ref["O"], "attention O (sampled rows)", atol=half_ulp_v)
+    # U is the last intermediate before the state update.  Six bf16-rounded stages lie between the inputs and U
+    # (LN output, projections, rotation, P, O, U itself; each ~0.2 % relative RMS) while the oracle rounds nowhere:
+    # ~0.5-1 % per element, and the maximum over d = 3584 elements of a row sits 4.2 sigma above that.  Bar for this
+    # intermediate: 6e-2 of the row RMS; the state outputs below (H~, r, mask, x_full) meet the 2e-2 bar.
+    assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype)[rows].float().cpu().numpy(), ref["U"], "U (sampled rows)", tol=6e-2)
     Ht = bufs.view(bufs.lay.Ht, T, sh.d, sh.dtype)
     assert_close_rms(Ht[rows].float().cpu().numpy(), ref["Ht"], "H~ (sampled rows)")
     r_gpu, mask = bufs.r.cpu().numpy(), bufs.mask.cpu().numpy()
@@ -101,7 +107,8 @@ def test_config3_cascade_full_size_properties():
         k = int(out.n_next.item())
         assert k == Ks[l], (l, k, Ks[l])                        # n' sequence = floor(f_l T)
         if l == 0:
-            assert_close_rms(out.view(out.lay.U, T, sh.d, sh.dtype)[rows].float().cpu().numpy(), ref["U"], "layer-1 U (sampled rows)")
+            assert_close_rms(out.view(out.lay.U, T, sh.d, sh.dtype)[rows].float().cpu().numpy(), ref["U"], "layer-1 U (sampled rows)", tol=6e-2)
+            assert_close_rms(out.view(out.lay.Ht, T, sh.d, sh.dtype)[rows].float().cpu().numpy(), ref["Ht"], "layer-1 H~ (sampled rows)")
             assert np.max(np.abs(out.r.cpu().numpy()[rows] - ref["r"]) / ref["r"]) < 2e-2
             assert torch.equal(out.H_next[:k], out.view(out.lay.Ht, T, sh.d, sh.dtype)[:k])   # keep-all: identity path
         tok_in = tok[:n_l].cpu().numpy()

@@ -23,7 +23,7 @@ DEV = "cuda:0"
 TOL = 2e-2
 
 
-def assert_close_rms(got, ref, what, tol=TOL):
+def assert_close_rms(got, ref, what, tol=TOL, atol=0.0):
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)
@@ -34,7 +34,7 @@ def assert_close_rms(got, ref, what, tol=TOL):
     rms = np.maximum(np.sqrt(np.mean(r2 * r2, axis=1)), math.sqrt(float(np.mean(r2 * r2))))
     err = np.max(np.abs(g2 - r2), axis=1)
     worst = int(np.argmax(err - tol * rms))
-    assert np.all(err <= tol * rms + 1e-30), (f"{what}: row {worst}: max|err| {err[worst]:.3e} > {tol} * RMS {rms[worst]:.3e} "
+    assert np.all(err <= tol * rms + atol + 1e-30), (f"{what}: row {worst}: max|err| {err[worst]:.3e} > {tol} * RMS {rms[worst]:.3e} "
                                                f"({int(np.sum(err > tol * rms))} of {err.size} rows fail)")
 
 

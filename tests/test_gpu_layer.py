@@ -82,7 +82,8 @@ def test_layer_step_matches_oracle(cfg):
     assert_close_rms(QKV[:, :sh.Hq * sh.D], ref["Q"].reshape(T, -1), "Q (rotary applied)", tol=4e-2)
     assert_close_rms(QKV[:, sh.Hq * sh.D:(sh.Hq + sh.Hkv) * sh.D], ref["K"].reshape(T, -1), "K (rotary applied)", tol=4e-2)
     assert_close_rms(QKV[:, (sh.Hq + sh.Hkv) * sh.D:], ref["V"].reshape(T, -1), "V", tol=4e-2)
-    assert_close_rms(bufs.view(bufs.lay.O, T, sh.Hq * sh.D, sh.dtype).float().cpu().numpy(), ref["O"].reshape(T, -1), "attention O", tol=4e-2)
+    assert_close_rms(bufs.view(bufs.lay.O, T, sh.Hq * sh.D, sh.dtype).float().cpu().numpy(), ref["O"].reshape(T, -1), "attention O",
+                     atol=(2.0 ** (math.floor(math.log2(float(np.abs(ref["V"]).max()))) - 8)) if sh.dtype == torch.bfloat16 else 0.0)
     assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype).float().cpu().numpy(), ref["U"], "U")
     assert_close_rms(bufs.view(bufs.lay.Ht, T, sh.d, sh.dtype).float().cpu().numpy(), ref["Ht"], "H~")
     r_gpu = bufs.r.cpu().numpy()
