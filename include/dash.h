@@ -45,6 +45,7 @@ extern "C" {
 #define DASH_ERR_WORKSPACE    3
 #define DASH_ERR_CUDA         4
 #define DASH_ERR_TIMEOUT      5
+#define DASH_ERR_TOO_LARGE    6
 
 typedef enum { DASH_F32 = 0, DASH_BF16 = 1 } dash_dtype;
 /* REL: ||U_t|| / ||H_t|| (the "relative" delta-attention of Fig. 1);
@@ -130,6 +131,29 @@ int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
                  const int32_t* tok_in, int32_t* tok_out,
                  int32_t* idx_out, int32_t* cu_out, int32_t* n_out_dev,
                  void* ws, size_t ws_bytes, void* stream);
+
+/* Same operation and arguments as dash_compact, for callers that cannot hand over a
+ * workspace because they are not allowed to allocate device memory at all: a serving
+ * loop whose device memory was handed out in full at start-up, or a plug-in whose host
+ * forbids allocation calls on its worker threads (they synchronise the device).  (The
+ * paper has no counterpart: it describes the method, not a memory policy.)
+ * The look-back scratch lives in a fixed array inside the library instead, which every
+ * GPU that loads the library holds until the process exits (256 KiB + 256 B).
+ *  - Limit: n <= DASH_COMPACT_STATIC_MAX_ROWS; larger inputs are rejected with
+ *    DASH_ERR_TOO_LARGE before anything is enqueued.
+ *  - Allocates nothing (no cudaMalloc / cudaFree, no allocating library routine); the
+ *    part of the array a call uses is cleared on `stream` before its kernel runs.
+ *  - The first call on a device looks up the device address of the array (with that
+ *    device current); make that first call before any stream capture begins.
+ *  - All calls on one device share the array and it keeps the last call's contents:
+ *    two calls whose kernels may overlap on the GPU (different streams) race.  Calls on
+ *    one stream are safe. */
+#define DASH_COMPACT_STATIC_MAX_ROWS (1 << 20)
+int dash_compact_static(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
+                        const dash_rows* rows /*host array*/, int n_rows,
+                        const int32_t* pos_in, int32_t* pos_out,
+                        const int32_t* tok_in, int32_t* tok_out,
+                        int32_t* idx_out, int32_t* cu_out, int32_t* n_out_dev, void* stream);
 
 /* dst_full[tok_index[i]] = src[i] for every i < n with sel[i] == which
  * (which: 0 halted rows, 1 active rows, 2 every row; sel may be NULL for 2).

@@ -35,6 +35,7 @@ extern "C" const char* dash_status_string(int status) {
         case DASH_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case DASH_ERR_CUDA: return "CUDA runtime error";
         case DASH_ERR_TIMEOUT: return "a device-side wait gave up";
+        case DASH_ERR_TOO_LARGE: return "input exceeds the fixed scratch of this entry point (use the variant that takes a workspace)";
         default: return "unknown status";
     }
 }

@@ -518,6 +518,39 @@ extern "C" int dash_scatter(const void* src, int64_t n, int64_t row_bytes, int64
     return DASH_OK;
 }
 
+// ---------------------------------------------------------------------------
+// Compaction for callers that may not allocate: the look-back scratch (ticket word
+// + one 64-bit state per 32-token tile) is a fixed array in the library image.
+// ---------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = 256 + (size_t)(DASH_COMPACT_STATIC_MAX_ROWS / 32 + 1) * 8;
+static __device__ __align__(256) unsigned char g_compact_scratch[(kStaticScratchBytes + 255) / 256 * 256];
+
+// Host code cannot use the array's name as a pointer (on the host it is only a handle for
+// the runtime): ask for its device address once per device, with that device current.
+static void* compact_scratch_ptr() {
+    static void* ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_compact_scratch) != cudaSuccess) return nullptr;
+        ptrs[dev] = p;
+    }
+    return ptrs[dev];
+}
+
+extern "C" int dash_compact_static(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
+                                   const dash_rows* rows, int n_rows,
+                                   const int32_t* pos_in, int32_t* pos_out, const int32_t* tok_in, int32_t* tok_out,
+                                   int32_t* idx_out, int32_t* cu_out, int32_t* n_out_dev, void* stream) {
+    if (n > DASH_COMPACT_STATIC_MAX_ROWS) return DASH_ERR_TOO_LARGE;
+    void* scratch = compact_scratch_ptr();
+    if (!scratch) return DASH_ERR_CUDA;
+    // same kernel and launch as dash_compact; it clears the part of the scratch it uses first
+    return dash_compact(mask, n, cu_in, S, rows, n_rows, pos_in, pos_out, tok_in, tok_out, idx_out, cu_out, n_out_dev,
+                        scratch, sizeof(g_compact_scratch), stream);
+}
+
 namespace dash {
 size_t select_ws_bytes(int64_t, int) { return 256; }
 size_t compact_ws_bytes_pub(int64_t n) { return compact_ws_bytes(n); }

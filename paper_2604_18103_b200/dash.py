@@ -27,8 +27,9 @@ LIB_PATH = os.path.join(_HERE, "libdash.so")
 EXPORTS = [
     "dash_status_string", "dash_check_status", "dash_keep_count", "dash_flops_per_layer", "dash_flops_speedup",
     "dash_delta_norm", "dash_select", "dash_compact", "dash_scatter", "dash_varlen_attention",
-    "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes",
+    "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes", "dash_compact_static",
 ]
+COMPACT_STATIC_MAX_ROWS = 1 << 20
 
 
 class Threshold(Structure):
@@ -80,6 +81,8 @@ def lib() -> ctypes.CDLL:
                                   c_void_p, c_void_p, c_size_t, c_void_p]
         L.dash_compact.argtypes = [c_void_p, c_int64, c_void_p, c_int, POINTER(Rows), c_int, c_void_p, c_void_p,
                                    c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.dash_compact_static.argtypes = [c_void_p, c_int64, c_void_p, c_int, POINTER(Rows), c_int, c_void_p, c_void_p,
+                                          c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.dash_scatter.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_int, c_void_p,
                                    c_void_p, c_int64, c_void_p]
         L.dash_varlen_attention.argtypes = [c_void_p] * 5 + [c_int64] * 4 + [c_void_p, c_int, c_int64, c_int64,
@@ -191,8 +194,13 @@ def dash_select(r: torch.Tensor, cu_seqlens: torch.Tensor, mode: int, tau: float
 # ---- step 3 ---------------------------------------------------------------------
 def dash_compact(mask: torch.Tensor, cu_in: torch.Tensor, rows: Sequence[torch.Tensor] = (),
                  rows_out: Optional[Sequence[torch.Tensor]] = None, pos_in: Optional[torch.Tensor] = None,
-                 tok_in: Optional[torch.Tensor] = None, want_idx: bool = True, ws: Optional[torch.Tensor] = None):
-    """Returns dict(idx, cu_out, n_out (device int32 [1]), rows (list), pos_out, tok_out); outputs are sized n."""
+                 tok_in: Optional[torch.Tensor] = None, want_idx: bool = True, ws: Optional[torch.Tensor] = None,
+                 outputs: Optional[dict] = None, static_scratch: bool = False):
+    """Returns dict(idx, cu_out, n_out (device int32 [1]), rows (list), pos_out, tok_out); outputs are sized n.
+
+    `outputs` may hand in preallocated idx / pos_out / tok_out / cu_out / n_out tensors.  With
+    static_scratch=True the call goes to dash_compact_static, the entry point for callers that
+    must not allocate: it takes no workspace and uses the library's fixed scratch array."""
     _dev(mask, cu_in)
     n = mask.numel()
     S = cu_in.numel() - 1
@@ -204,11 +212,17 @@ def dash_compact(mask: torch.Tensor, cu_in: torch.Tensor, rows: Sequence[torch.T
         rb = x.shape[1] * x.element_size() if x.dim() > 1 else x.element_size()
         rb = int(x[0].numel() * x.element_size()) if x.shape[0] > 0 else rb
         arr[i] = Rows(x.data_ptr(), y.data_ptr(), rb, x.stride(0) * x.element_size(), y.stride(0) * y.element_size())
-    idx = torch.empty(n, dtype=torch.int32, device=dev) if want_idx else None
-    pos_out = torch.empty(n, dtype=torch.int32, device=dev) if pos_in is not None else None
-    tok_out = torch.empty(n, dtype=torch.int32, device=dev) if tok_in is not None else None
-    cu_out = torch.empty(S + 1, dtype=torch.int32, device=dev)
-    n_out = torch.empty(1, dtype=torch.int32, device=dev)
+    o = outputs or {}
+    idx = o.get("idx", torch.empty(n, dtype=torch.int32, device=dev) if want_idx else None)
+    pos_out = o.get("pos_out", torch.empty(n, dtype=torch.int32, device=dev) if pos_in is not None else None)
+    tok_out = o.get("tok_out", torch.empty(n, dtype=torch.int32, device=dev) if tok_in is not None else None)
+    cu_out = o.get("cu_out", torch.empty(S + 1, dtype=torch.int32, device=dev))
+    n_out = o.get("n_out", torch.empty(1, dtype=torch.int32, device=dev))
+    if static_scratch:
+        st = lib().dash_compact_static(_p(mask), n, _p(cu_in), S, arr, len(rows), _p(pos_in), _p(pos_out), _p(tok_in),
+                                       _p(tok_out), _p(idx), _p(cu_out), _p(n_out), _stream())
+        _check(st, "dash_compact_static")
+        return {"idx": idx, "cu_out": cu_out, "n_out": n_out, "rows": list(rows_out), "pos_out": pos_out, "tok_out": tok_out}
     if ws is None:
         ws = workspace(dash_workspace_bytes(WS_COMPACT, n, S), dev)
     st = lib().dash_compact(_p(mask), n, _p(cu_in), S, arr, len(rows), _p(pos_in), _p(pos_out), _p(tok_in), _p(tok_out),
