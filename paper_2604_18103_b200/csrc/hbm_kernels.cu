@@ -223,10 +223,14 @@ select_keep_count_kernel(const float* __restrict__ r, const int32_t* __restrict_
 }
 
 // ---------------------------------------------------------------------------
-// step 3: compaction.  Single pass: each CTA takes a tile of TILE tokens
-// (ticket order), ballots its mask, publishes the tile count, finds its output
-// base by decoupled look-back over the preceding tiles, then its warps move the
-// tile's active rows with 128-bit accesses.
+// step 3: compaction.  Single pass: each CTA takes a tile of TILE tokens, ballots
+// its mask, finds its output base, then its 16 warps move the tile's active rows
+// in 4 KB pieces (128-bit accesses, 8 per lane in flight).
+// Output base of a tile = number of active tokens before it:
+//  - DIRECT (small inputs): counted straight from the mask bytes in front of the
+//    tile (a few KB from L2) -- no scratch, no ordering between CTAs;
+//  - otherwise: ticketed tiles publish their counts and look back over the
+//    preceding tiles (decoupled look-back, bounded spin).
 // ---------------------------------------------------------------------------
 struct RowStreams {
     const char* src[DASH_MAX_ROW_STREAMS];
@@ -237,6 +241,8 @@ struct RowStreams {
 };
 
 constexpr unsigned long long kFlagAgg = 1ull << 32, kFlagPrefix = 2ull << 32;
+constexpr int kCompactThreads = 512;
+constexpr int kPieceBytes = 4096;                       // one warp moves one piece at a time
 
 __device__ __forceinline__ unsigned long long ld_state(const unsigned long long* p) {
     unsigned long long v;
@@ -246,24 +252,32 @@ __device__ __forceinline__ unsigned long long ld_state(const unsigned long long*
 __device__ __forceinline__ void st_state(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
+__device__ __forceinline__ int nonzero_bytes(uint32_t w) { return __popc(__vcmpne4(w, 0u)) >> 3; }
 
-template <int TILE>
-__global__ void __launch_bounds__(256)
+template <int TILE, bool DIRECT>
+__global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(const uint8_t* __restrict__ mask, int64_t n_upper, const int32_t* __restrict__ cu_in, int S,
                RowStreams rs, const int32_t* __restrict__ pos_in, int32_t* __restrict__ pos_out,
                const int32_t* __restrict__ tok_in, int32_t* __restrict__ tok_out,
                int32_t* __restrict__ idx_out, int32_t* __restrict__ cu_out, int32_t* __restrict__ n_out_dev,
-               unsigned long long* tile_state, unsigned int* ticket, int* status) {
+               unsigned long long* tile_state, unsigned int* ticket, int* status, int mask_vec16) {
     constexpr int NW = TILE / 32;                       // warps that ballot
+    constexpr int NWARPS = kCompactThreads / 32;
     __shared__ unsigned int s_ballot[NW];
     __shared__ int s_wprefix[NW + 1];
     __shared__ int s_src[TILE];
     __shared__ int s_base;
+    __shared__ int s_part[NWARPS];
     __shared__ unsigned int s_tile;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
-    __syncthreads();
-    const int tile = (int)s_tile;
+    int tile;
+    if (DIRECT) {
+        tile = (int)blockIdx.x;
+    } else {
+        if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
+        __syncthreads();
+        tile = (int)s_tile;
+    }
     int64_t n = cu_in[S];
     if (n > n_upper) n = n_upper;
     const int64_t t_start = (int64_t)tile * TILE;
@@ -278,6 +292,22 @@ compact_kernel(const uint8_t* __restrict__ mask, int64_t n_upper, const int32_t*
         unsigned int bal = __ballot_sync(0xffffffffu, my);
         if (lane == 0) s_ballot[warp] = bal;
     }
+    if (DIRECT) {
+        // active tokens in front of this tile, straight from the mask (t_start is a multiple of 32)
+        int cnt = 0;
+        if (mask_vec16) {
+            const uint4* mv = reinterpret_cast<const uint4*>(mask);
+            for (int64_t v = threadIdx.x; v < (t_start >> 4); v += kCompactThreads) {
+                const uint4 w = ld_nc_v4(mv + v);
+                cnt += nonzero_bytes(w.x) + nonzero_bytes(w.y) + nonzero_bytes(w.z) + nonzero_bytes(w.w);
+            }
+        } else {
+            for (int64_t t = threadIdx.x; t < t_start; t += kCompactThreads) cnt += (mask[t] != 0);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if (lane == 0) s_part[warp] = cnt;
+    }
     __syncthreads();
     if (warp == 0) {
         int c = (lane < NW) ? __popc(s_ballot[lane]) : 0;
@@ -290,11 +320,16 @@ compact_kernel(const uint8_t* __restrict__ mask, int64_t n_upper, const int32_t*
         if (lane < NW) s_wprefix[lane] = inc - c;
         const int agg = __shfl_sync(0xffffffffu, inc, 31);
         if (lane == 0) s_wprefix[NW] = agg;
-        // publish this tile's count, then look back
         int base = 0;
-        if (tile == 0) {
+        if (DIRECT) {
+            int v = (lane < NWARPS) ? s_part[lane] : 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            base = v;
+        } else if (tile == 0) {
             if (lane == 0) st_state(&tile_state[0], kFlagPrefix | (unsigned int)agg);
         } else {
+            // publish this tile's count, then look back
             if (lane == 0) st_state(&tile_state[tile], kFlagAgg | (unsigned int)agg);
             int look = tile - 1;
             bool done = false, timed_out = false;
@@ -351,14 +386,24 @@ compact_kernel(const uint8_t* __restrict__ mask, int64_t n_upper, const int32_t*
         }
     }
     __syncthreads();
-    // move the rows
-    const int nwarps = blockDim.x >> 5;
+    // move the rows: the tile's (row, piece) items are dealt round-robin to the warps, across all row tensors
+    int first_warp = 0;                                 // warp that takes item 0 of the current tensor
     for (int q = 0; q < rs.count; ++q) {
-        for (int k = warp; k < count; k += nwarps) {
-            const char* src = rs.src[q] + (int64_t)s_src[k] * rs.src_ld[q];
-            char* dst = rs.dst[q] + (int64_t)(base + k) * rs.dst_ld[q];
-            if (rs.vec16[q]) warp_copy_row16(src, dst, rs.row_bytes[q], lane);
-            else warp_copy_row4(src, dst, rs.row_bytes[q], lane);
+        const int64_t rb = rs.row_bytes[q];
+        if (rs.vec16[q]) {
+            const int pieces = (int)((rb + kPieceBytes - 1) / kPieceBytes);
+            const int items = count * pieces;
+            for (int it = (warp - first_warp + NWARPS) % NWARPS; it < items; it += NWARPS) {
+                const int k = it / pieces, pc = it - k * pieces;
+                const int64_t off = (int64_t)pc * kPieceBytes;
+                const int64_t len = (rb - off < kPieceBytes) ? rb - off : kPieceBytes;
+                warp_copy_row16(rs.src[q] + (int64_t)s_src[k] * rs.src_ld[q] + off, rs.dst[q] + (int64_t)(base + k) * rs.dst_ld[q] + off, len, lane);
+            }
+            first_warp = (first_warp + items) % NWARPS;
+        } else {
+            for (int k = (warp - first_warp + NWARPS) % NWARPS; k < count; k += NWARPS)
+                warp_copy_row4(rs.src[q] + (int64_t)s_src[k] * rs.src_ld[q], rs.dst[q] + (int64_t)(base + k) * rs.dst_ld[q], rb, lane);
+            first_warp = (first_warp + count) % NWARPS;
         }
     }
 }
@@ -453,6 +498,8 @@ static int compact_tile_for(int64_t n) {
     if (n / 64 >= want) return 64;
     return 32;
 }
+// up to this many rows the output base of a tile is counted straight from the mask (no scratch, no look-back)
+constexpr int64_t kCompactDirectMaxRows = 32768;
 
 static size_t compact_ws_bytes(int64_t n) {
     int64_t tiles = (n + 31) / 32 + 1;
@@ -484,19 +531,30 @@ extern "C" int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in
     cudaStream_t st = (cudaStream_t)stream;
     const int TILE = compact_tile_for(n);
     const int tiles = (int)((n + TILE - 1) / TILE) > 0 ? (int)((n + TILE - 1) / TILE) : 1;
+    const bool direct = n <= kCompactDirectMaxRows;
     unsigned int* ticket = (unsigned int*)ws;
     unsigned long long* state = (unsigned long long*)((char*)ws + 256);
-    DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)tiles * 8, st));
+    if (!direct) DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)tiles * 8, st));
     int* status = status_word_ptr();
     if (!status) return DASH_ERR_CUDA;
-#define DASH_LAUNCH_COMPACT(T)                                                                                    \
-    compact_kernel<T><<<tiles, 256, 0, st>>>(mask, n, cu_in, S, rs, pos_in, pos_out, tok_in, tok_out, idx_out, \
-                                             cu_out, n_out_dev, state, ticket, status)
-    switch (TILE) {
-        case 256: DASH_LAUNCH_COMPACT(256); break;
-        case 128: DASH_LAUNCH_COMPACT(128); break;
-        case 64: DASH_LAUNCH_COMPACT(64); break;
-        default: DASH_LAUNCH_COMPACT(32); break;
+    const int mask_vec16 = aligned16(mask) ? 1 : 0;
+#define DASH_LAUNCH_COMPACT(T, DIRECT)                                                                                       \
+    compact_kernel<T, DIRECT><<<tiles, kCompactThreads, 0, st>>>(mask, n, cu_in, S, rs, pos_in, pos_out, tok_in, tok_out, \
+                                                                 idx_out, cu_out, n_out_dev, state, ticket, status, mask_vec16)
+    if (direct) {
+        switch (TILE) {
+            case 256: DASH_LAUNCH_COMPACT(256, true); break;
+            case 128: DASH_LAUNCH_COMPACT(128, true); break;
+            case 64: DASH_LAUNCH_COMPACT(64, true); break;
+            default: DASH_LAUNCH_COMPACT(32, true); break;
+        }
+    } else {
+        switch (TILE) {
+            case 256: DASH_LAUNCH_COMPACT(256, false); break;
+            case 128: DASH_LAUNCH_COMPACT(128, false); break;
+            case 64: DASH_LAUNCH_COMPACT(64, false); break;
+            default: DASH_LAUNCH_COMPACT(32, false); break;
+        }
     }
 #undef DASH_LAUNCH_COMPACT
     DASH_CUDA_TRY(cudaGetLastError());
