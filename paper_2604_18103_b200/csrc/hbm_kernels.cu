@@ -491,12 +491,13 @@ extern "C" int dash_select(const float* r, int64_t n, const int32_t* cu_seqlens,
     return DASH_OK;
 }
 
+// Tokens per CTA.  Small tiles keep the CTAs balanced when the active rows cluster (a packed batch whose
+// image blocks halt almost entirely while its text blocks stay); larger ones only bound the look-back chain.
 static int compact_tile_for(int64_t n) {
-    const int64_t want = 2LL * sm_count();
-    if (n / 256 >= want) return 256;
-    if (n / 128 >= want) return 128;
-    if (n / 64 >= want) return 64;
-    return 32;
+    if (n <= 16384) return 32;
+    if (n <= 262144) return 64;
+    if (n <= 1048576) return 128;
+    return 256;
 }
 // up to this many rows the output base of a tile is counted straight from the mask (no scratch, no look-back)
 constexpr int64_t kCompactDirectMaxRows = 32768;
