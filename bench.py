@@ -229,8 +229,8 @@ def setup_block_step(args, dash, dev, rank):
     name = "configs[0]: single fp32 layer, hidden 256, 4 heads of 64" if args.workload == "cfg1" else "configs[1]: Qwen2.5-7B-shaped single layer, bf16"
     return {
         "workload": f"{name}, batch 1, seq {T}, threshold at the {int(w.rho * 100)}th percentile ({n_active} of {T} tokens stay active)",
-        "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 6,
-        "launch_note": "per step: rmsnorm, rope, attention, delta_norm(+residual+threshold), scatter, compact "
+        "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 7,
+        "launch_note": "per step: rmsnorm, rope, attention plan, attention, delta_norm(+residual+threshold), scatter, compact "
                        "(+2 cuBLASLt GEMMs that are not this library's kernels)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(*host_out),
         "extra": {"n_active_after": n_active, "tau": tau},
@@ -301,7 +301,7 @@ def setup_cascade(args, dash, dev, rank):
     Kt = QKV[:, sh.Hq * sh.D:(sh.Hq + sh.Hkv) * sh.D].view(T, sh.Hkv, sh.D)
     V = QKV[:, (sh.Hq + sh.Hkv) * sh.D:].view(T, sh.Hkv, sh.D)
     Obuf = A.view(A.lay.O, T, sh.Hq * sh.D, sh.dtype).view(T, sh.Hq, sh.D)
-    attn_ws = dash.workspace(256, dev)
+    attn_ws = dash.workspace(dash.dash_workspace_bytes(dash.WS_ATTENTION, T, S, sh.Hq, sh.Hkv, sh.D), dev)
     U, Ht = A.view(A.lay.U, T, sh.d, sh.dtype), A.view(A.lay.Ht, T, sh.d, sh.dtype)
     cws = dash.workspace(dash.dash_workspace_bytes(dash.WS_COMPACT, T, S), dev)
     mask2 = wl.random_mask(T, 0.9, seed=7).to(dev)         # the second layer's keep ratio, for the stand-alone compaction timing
@@ -309,8 +309,8 @@ def setup_cascade(args, dash, dev, rank):
     fl_all = sum(attention_flops([0, n], sh.Hq, sh.D) for n in n_in)
     return {
         "workload": f"configs[2]: cascade of {Lr} Qwen2.5-7B-shaped layers, bf16, batch 1, seq {T}, tokens entering the layers {n_in}, "
-                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 6 * Lr,
-        "launch_note": f"{Lr} block steps of 6 kernels each (+2 cuBLASLt GEMMs per block step)",
+                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 7 * Lr,
+        "launch_note": f"{Lr} block steps of 7 kernels each (+2 cuBLASLt GEMMs per block step)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(x_full_h, tok_h, cu_h),
         "extra": {"tokens_entering_layers": n_in, "active_after_last": got, "attention_flops_per_step": fl_all,
                   "value_counts": "tokens entering each of the 8 layers, summed"},
@@ -338,7 +338,7 @@ def setup_sparse(args, dash, dev, rank):
     o = {"pos_out": torch.empty_like(pos), "tok_out": torch.empty_like(pos), "cu_out": torch.empty_like(cu), "n_out": torch.empty(1, dtype=torch.int32, device=dev)}
     O = torch.empty(T, sh.Hq, sh.D, dtype=sh.dtype, device=dev)
     cws = dash.workspace(dash.dash_workspace_bytes(dash.WS_COMPACT, T, S), dev)
-    attn_ws = dash.workspace(256, dev)
+    attn_ws = dash.workspace(dash.dash_workspace_bytes(dash.WS_ATTENTION, T, S, sh.Hq, sh.Hkv, sh.D), dev)
     O_h, tok_h, cu_h, r_h = _pin(torch.empty(T, sh.Hq * sh.D, dtype=sh.dtype)), _pin(torch.empty(T, dtype=torch.int32)), _pin(torch.empty(S + 1, dtype=torch.int32)), _pin(torch.empty(T))
 
     def h2d():
@@ -381,12 +381,12 @@ def setup_sparse(args, dash, dev, rank):
     return {
         "workload": f"{which}; Qwen2.5-7B layer shape, bf16; score+threshold -> compaction of H~,Q,K,V -> causal GQA attention over the "
                     f"{k} active of {T} tokens (compacted lengths {lens_out})",
-        "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 3,
-        "launch_note": "per step: delta_norm(+residual+threshold), compact (4 row tensors), attention (grid sized by the longest entering sequence)",
+        "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 4,
+        "launch_note": "per step: delta_norm(+residual+threshold), compact (4 row tensors; + a memset of its look-back scratch), attention plan, attention",
         "h2d_bytes": _bytes(*host.values(), pos_host, cu_host), "d2h_bytes": _bytes(O_h, tok_h, cu_h, r_h),
         "extra": {"n_active_after": k, "tau": state["tau"]},
         "attn": (lambda: attn()), "attn_flops": attention_flops(cu_out, sh.Hq, sh.D),
-        "attn_name": f"attention_kernel<{sh.D}> over the compacted set (grid sized by the true longest sequence)",
+        "attn_name": f"attention_kernel<{sh.D}> over the compacted set",
         "norm": norm, "norm_bytes": T * (3 * sh.d * es + 5),
         "compact": compact, "compact_bytes": k * (2 * row_b + 16) + T * 9, "compact_rows": k, "row_bytes": row_b,
     }

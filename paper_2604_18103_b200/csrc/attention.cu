@@ -1,7 +1,9 @@
 // Causal grouped-query attention over a packed (varlen) batch of active tokens,
 // on tcgen05 tensor cores with TMEM accumulators, operands staged by TMA.
 //
-// Work unit (one CTA): 128 consecutive query rows of one head of one sequence.
+// Work item: 128 consecutive query rows of one head of one sequence.  A small plan kernel lists the
+// items that exist (from cu_seqlens, on the device), heaviest first; persistent CTAs (two per SM) take
+// them by ticket, so that no CTA is spent on query tiles that a shorter sequence does not have.
 // Thread roles: warps 0-3 own one query row each (TMEM lane = row) and do the
 // online softmax; warp 4 allocates TMEM and its lane 0 issues every TMA load and
 // every tcgen05.mma.  Two CTAs share an SM (256 TMEM columns and < 113 KB of
@@ -81,7 +83,60 @@ struct AttnParams {
     float* lse;             // [Hq, n] or null
     int64_t n;
     int* status;
+    const int2* plan;           // (sequence, query tile) of every item group, heaviest first; Hq items (heads) per entry
+    const int* n_items;         // device: entries * Hq
+    unsigned int* ticket;       // device: next item to hand out
 };
+
+// ---- plan: which (sequence, query tile) pairs exist, ordered by falling number of key blocks ----
+__global__ void __launch_bounds__(1024)
+attention_plan_kernel(const int32_t* __restrict__ cu, int S, int Hq, int2* __restrict__ plan, int* __restrict__ n_items,
+                      unsigned int* __restrict__ ticket, int64_t max_entries) {
+    __shared__ int s_warp[33];
+    __shared__ int s_max;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_max = 0;
+    __syncthreads();
+    int mx = 0;
+    for (int s = tid; s < S; s += blockDim.x) mx = max(mx, (cu[s + 1] - cu[s] + kBM - 1) / kBM);
+    atomicMax(&s_max, mx);
+    __syncthreads();
+    const int max_nq = s_max;
+    int64_t offset = 0;
+    for (int top = max_nq - 1; top >= 0; top -= (int)blockDim.x) {
+        const int qt = top - tid;                           // thread 0 takes the heaviest level of this chunk
+        int cnt = 0;
+        if (qt >= 0)
+            for (int s = 0; s < S; ++s) cnt += ((cu[s + 1] - cu[s] + kBM - 1) / kBM > qt);
+        // exclusive scan over the block
+        const int lane = tid & 31, w = tid >> 5;
+        int inc = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+        if (lane == 31) s_warp[w] = inc;
+        __syncthreads();
+        if (w == 0) {
+            int x = s_warp[lane], xi = x;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xffffffffu, xi, o); if (lane >= o) xi += t; }
+            s_warp[lane] = xi - x;
+            if (lane == 31) s_warp[32] = xi;
+        }
+        __syncthreads();
+        int64_t k = offset + s_warp[w] + inc - cnt;
+        const int chunk_total = s_warp[32];
+        if (qt >= 0)
+            for (int s = 0; s < S; ++s)
+                if ((cu[s + 1] - cu[s] + kBM - 1) / kBM > qt) { if (k < max_entries) plan[k] = make_int2(s, qt); ++k; }
+        offset += chunk_total;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        if (offset > max_entries) offset = max_entries;     // cannot happen for cu_seqlens[S] <= n; keeps every read in bounds
+        *n_items = (int)(offset * Hq);
+        *ticket = 0u;
+    }
+}
 
 template <int D>
 struct AttnSmem {
@@ -108,18 +163,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     volatile uint32_t* abort_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 68);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-    // heavy (late) query tiles first; the heads of one KV group run together
-    const int per_tile = p.Hq * p.S;
-    const int qt = p.n_qtiles - 1 - (int)(blockIdx.x / per_tile);
-    const int rem = (int)(blockIdx.x % per_tile);
-    const int h = rem % p.Hq, s = rem / p.Hq;
-    const int kvh = h / (p.Hq / p.Hkv);
-    const int seq_a = p.cu[s], seq_b = p.cu[s + 1];
-    const int len = seq_b - seq_a;
-    const int q0 = qt * kBM;
-    if (q0 >= len) return;                                   // uniform for the CTA: nothing allocated yet
-    const int nblk = qt + 1;                                 // causal: key blocks 0..qt
+    volatile int* item_gen = reinterpret_cast<volatile int*>(smem_gen + L::kBars + 72);
 
     if (warp == 4) {
         if (lane == 0) {
@@ -142,6 +186,26 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 
     constexpr uint32_t idesc_s = idesc_bf16_f32(kBM, kBN, false, false);
     constexpr uint32_t idesc_o = idesc_bf16_f32(kBM, D, false, true);
+    const int n_items = *p.n_items;
+    const int G = p.Hq / p.Hkv;
+    // Barrier phases run on across the items of this CTA: blk0 = key blocks of its earlier items, items_done = their number.
+    uint32_t blk0 = 0, items_done = 0;
+
+    for (;;) {
+    if (tid == 0) *item_gen = (int)atomicAdd(p.ticket, 1u);
+    __syncthreads();
+    const int item = *item_gen;
+    if (item >= n_items || *abort_gen) break;
+    tc_fence_after();
+    // the heads of one KV group run next to each other, so their K/V tiles are shared through L2
+    const int2 e = p.plan[item / p.Hq];
+    const int h = item % p.Hq, s = e.x, qt = e.y;
+    const int kvh = h / G;
+    const int seq_a = p.cu[s], seq_b = p.cu[s + 1];
+    const int len = seq_b - seq_a;
+    const int q0 = qt * kBM;
+    const int nblk = qt + 1;                                 // causal: key blocks 0..qt
+    const uint32_t qph = items_done & 1;
 
     if (warp == 4) {
         if (lane == 0) {
@@ -161,10 +225,10 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 }
                 tc_commit(bar_s);
             };
-            ok = mbar_wait(bar_q, 0, kWaitCycles) && mbar_wait(bar_k, 0, kWaitCycles);
+            ok = mbar_wait(bar_q, qph, kWaitCycles) && mbar_wait(bar_k, blk0 & 1, kWaitCycles);
             if (ok) issue_s();
             for (int j = 0; j < nblk && ok; ++j) {
-                const uint32_t ph = j & 1;
+                const uint32_t ph = (blk0 + j) & 1;
                 // S_j done: the K buffer is free for the next block
                 ok = mbar_wait(bar_s, ph, kWaitCycles);
                 if (!ok) break;
@@ -189,7 +253,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 // S_{j+1} goes into the pipe right behind PV_j: tcgen05.mma of one thread execute in issue
                 // order, so PV_j has read P_j before S_{j+1} overwrites the columns they share
                 if (j + 1 < nblk) {
-                    ok = mbar_wait(bar_k, (j + 1) & 1, kWaitCycles);
+                    ok = mbar_wait(bar_k, (blk0 + j + 1) & 1, kWaitCycles);
                     if (!ok) break;
                     issue_s();
                 }
@@ -211,7 +275,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         for (int j = 0; j < nblk; ++j) {
-            const uint32_t ph = j & 1;
+            const uint32_t ph = (blk0 + j) & 1;
             ok = mbar_wait(bar_s, ph, kWaitCycles);
             if (!ok || *abort_gen) { ok = false; break; }
             tc_fence_after();
@@ -246,7 +310,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 // O still holds the previous blocks' sum scaled by the old reference max
                 const bool need = __any_sync(0xffffffffu, grow);
                 if (need) {
-                    ok = mbar_wait(bar_o, (j - 1) & 1, kWaitCycles);
+                    ok = mbar_wait(bar_o, (blk0 + j - 1) & 1, kWaitCycles);
                     if (!ok) break;
                     tc_fence_after();
                     // rare path (the reference max moves in the first blocks only): small chunks, not
@@ -305,7 +369,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             l = l * alpha + ((sumA.x + sumA.y) + (sumB.x + sumB.y));
             m = m_new;
         }
-        if (ok) ok = mbar_wait(bar_o, (nblk - 1) & 1, kWaitCycles);
+        if (ok) ok = mbar_wait(bar_o, (blk0 + nblk - 1) & 1, kWaitCycles);
         if (ok && !*abort_gen) {
             tc_fence_after();
             const float inv = 1.0f / l;
@@ -341,8 +405,15 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             }
             if (row_valid && p.lse) p.lse[(int64_t)h * p.n + grow] = m * p.scale + logf(l);
         } else if (!ok && lane == 0) {
+            *abort_gen = 1;
             atomicExch(p.status, DASH_ERR_TIMEOUT);
         }
+    }
+    // end of the item: O has been read out, every tile buffer is free
+    tc_fence_before();
+    __syncthreads();
+    blk0 += (uint32_t)nblk;
+    ++items_done;
     }
     tc_fence_before();
     __syncthreads();
@@ -364,10 +435,14 @@ __global__ void f32_to_bf16_rows_kernel(const float* __restrict__ src, int64_t l
     }
 }
 
+// workspace: [0,256) ticket + item count; then the plan (one int2 per existing (sequence, query tile));
+// then, for fp32 tensors, their bf16 copies
+static size_t plan_entries(int64_t n, int S) { return (size_t)(n / kBM) + (size_t)S + 1; }
+static size_t plan_bytes(int64_t n, int S) { return align_up(plan_entries(n, S) * sizeof(int2), 256); }
 size_t attention_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt) {
-    (void)S;
-    if (dt == DASH_BF16) return 256;
-    return align_up((size_t)n * (Hq + 2 * Hkv) * D * 2, 256) + 256;
+    size_t b = 256 + plan_bytes(n, S);
+    if (dt != DASH_BF16) b += align_up((size_t)n * (Hq + 2 * Hkv) * D * 2, 256);
+    return b;
 }
 
 template <int D, bool OUT_F32>
@@ -409,9 +484,9 @@ extern "C" int dash_varlen_attention(const void* Q, const void* K, const void* V
 
     const void *q = Q, *k = K, *v = V;
     int64_t lq = ldq, lk = ldk, lv = ldv;
+    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < attention_ws_bytes(n, S, Hq, Hkv, D, dt)) return DASH_ERR_WORKSPACE;
     if (dt == DASH_F32) {
-        if (!ws || ((uintptr_t)ws % 256) || ws_bytes < attention_ws_bytes(n, S, Hq, Hkv, D, dt)) return DASH_ERR_WORKSPACE;
-        __nv_bfloat16* qb = (__nv_bfloat16*)ws;
+        __nv_bfloat16* qb = (__nv_bfloat16*)((char*)ws + 256 + plan_bytes(n, S));
         __nv_bfloat16* kb = qb + (size_t)n * Hq * D;
         __nv_bfloat16* vb = kb + (size_t)n * Hkv * D;
         const int cap = sm_count() * 8;
@@ -440,8 +515,16 @@ extern "C" int dash_varlen_attention(const void* Q, const void* K, const void* V
     p.O = O; p.ldo = ldo; p.lse = lse; p.n = n;
     p.status = status_word_ptr();
     if (!p.status) return DASH_ERR_CUDA;
-    const int64_t grid64 = (int64_t)p.n_qtiles * Hq * S;
-    if (grid64 > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
+    p.ticket = (unsigned int*)ws;
+    p.n_items = (const int*)((char*)ws + 4);
+    p.plan = (const int2*)((char*)ws + 256);
+    if ((int64_t)plan_entries(n, S) * Hq > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
+    attention_plan_kernel<<<1, 1024, 0, st>>>(cu_seqlens, S, Hq, (int2*)((char*)ws + 256), (int*)((char*)ws + 4), (unsigned int*)ws,
+                                              (int64_t)plan_entries(n, S));
+    DASH_CUDA_TRY(cudaGetLastError());
+    // persistent CTAs, two per SM, never more than there can be items
+    int64_t grid64 = (int64_t)p.n_qtiles * Hq * S;
+    if (grid64 > 2LL * sm_count()) grid64 = 2LL * sm_count();
     const int grid = (int)grid64;
     if (D == 128) return dt == DASH_F32 ? launch_attention<128, true>(mq, mk, mv, p, grid, st) : launch_attention<128, false>(mq, mk, mv, p, grid, st);
     return dt == DASH_F32 ? launch_attention<64, true>(mq, mk, mv, p, grid, st) : launch_attention<64, false>(mq, mk, mv, p, grid, st);
