@@ -229,9 +229,9 @@ def setup_block_step(args, dash, dev, rank):
     name = "configs[0]: single fp32 layer, hidden 256, 4 heads of 64" if args.workload == "cfg1" else "configs[1]: Qwen2.5-7B-shaped single layer, bf16"
     return {
         "workload": f"{name}, batch 1, seq {T}, threshold at the {int(w.rho * 100)}th percentile ({n_active} of {T} tokens stay active)",
-        "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 7,
-        "launch_note": "per step: rmsnorm, rope, attention plan, attention, delta_norm(+residual+threshold), scatter, compact "
-                       "(+2 cuBLASLt GEMMs that are not this library's kernels)",
+        "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 5,
+        "launch_note": "per step: rmsnorm, rope, attention plan, attention, fused tail (score + residual + threshold + scatter + compaction) "
+                       "(+2 cuBLASLt GEMMs and a memset that are not this library's kernels)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(*host_out),
         "extra": {"n_active_after": n_active, "tau": tau},
         "attn": (lambda: dash.dash_varlen_attention(Q, Kt, V, cu, T, O=Obuf, ws=attn_ws)), "attn_flops": attention_flops(w.cu.tolist(), sh.Hq, sh.D),
@@ -309,8 +309,8 @@ def setup_cascade(args, dash, dev, rank):
     fl_all = sum(attention_flops([0, n], sh.Hq, sh.D) for n in n_in)
     return {
         "workload": f"configs[2]: cascade of {Lr} Qwen2.5-7B-shaped layers, bf16, batch 1, seq {T}, tokens entering the layers {n_in}, "
-                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 7 * Lr,
-        "launch_note": f"{Lr} block steps of 7 kernels each (+2 cuBLASLt GEMMs per block step)",
+                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 5 * Lr,
+        "launch_note": f"{Lr} block steps of 5 kernels each (+2 cuBLASLt GEMMs per block step)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(x_full_h, tok_h, cu_h),
         "extra": {"tokens_entering_layers": n_in, "active_after_last": got, "attention_flops_per_step": fl_all,
                   "value_counts": "tokens entering each of the 8 layers, summed"},

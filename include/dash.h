@@ -198,7 +198,10 @@ typedef struct {
 } dash_layer_cfg;
 
 /* Byte offsets of the intermediates inside the workspace of dash_layer_step
- * (for inspection by tests and tools). */
+ * (for inspection by tests and tools).  Ht (H~ = H + U) is only written when the
+ * halting rule is KEEP_COUNT or scatter_which is 0; with the threshold rule and
+ * scatter_which = 2 the score, the residual, the scatter and the compaction run as
+ * one pass that writes H~ straight to x_full and H_next. */
 typedef struct {
     size_t Hn, QKV, O, U, Ht, scratch, total;
 } dash_layer_ws_layout;
@@ -210,7 +213,8 @@ int dash_layer_workspace(const dash_layer_cfg* cfg, int64_t n, int S, dash_layer
  * causal attention -> output projection U -> r, H~ = H + U -> halting rule ->
  * scatter of H~ into x_full [T, d] -> compaction of the tokens that stay
  * active into H_next / tok_index_next / pos_next / cu_next / n_next_dev.
- * r_out fp32 [n], mask_out u8 [n].  No host synchronisation. */
+ * r_out fp32 [n], mask_out u8 [n].  No host synchronisation.  x_full must not
+ * overlap H_in (unless tok_index_in is the identity and the rows coincide). */
 int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, const int32_t* tok_index_in,
                     const int32_t* pos_in, const int32_t* cu_in, int S, int64_t n, int64_t max_seqlen,
                     void* x_full, void* H_next, int32_t* tok_index_next, int32_t* pos_next,

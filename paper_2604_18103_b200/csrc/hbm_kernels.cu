@@ -422,6 +422,166 @@ scatter_kernel(const char* __restrict__ src, int64_t n, int64_t row_bytes, int64
     }
 }
 
+// ---------------------------------------------------------------------------
+// Steps 1-3 of the block step in one pass (threshold rule, every row's H~ written to the full-length
+// buffer): per tile of 32 tokens the 16 warps form r, the keep decision and H~ = H + U, stream H~ to
+// x_full[tok[row]], then the tile finds its output base by decoupled look-back and copies its active
+// rows (just written, still in L2) into the next block's packed buffer.  Reads U and H once, writes
+// x_full and H_next once: no separate scatter and compaction passes over H~.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint4 ld_cg_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+
+struct TailArgs {
+    const char* U; const char* H; int64_t ldU_b, ldH_b; int nvec; int mode; float eps;
+    float tau; int keep_first, keep_last; const int32_t* cu_in; int S;
+    const int32_t* tok_in; const int32_t* pos_in;
+    char* x_full; int64_t ldx_b; char* H_next; int64_t ldn_b;
+    float* r_out; uint8_t* mask_out; int32_t* tok_next; int32_t* pos_next; int32_t* cu_next; int32_t* n_next;
+    unsigned long long* tile_state; unsigned int* ticket; int* status;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(kCompactThreads, 2)
+delta_tail_kernel(const TailArgs a, int64_t n_upper) {
+    constexpr int TILE = 32, NWARPS = kCompactThreads / 32, RPW = TILE / NWARPS;   // 2 rows per warp
+    __shared__ int s_keep[TILE];
+    __shared__ int s_src[TILE];
+    __shared__ int s_base, s_count;
+    __shared__ unsigned int s_tile, s_ballot;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_tile = atomicAdd(a.ticket, 1u);
+    __syncthreads();
+    const int tile = (int)s_tile;
+    int64_t n = a.cu_in[a.S];
+    if (n > n_upper) n = n_upper;
+    const int64_t t_start = (int64_t)tile * TILE;
+    if (t_start >= n && tile != 0) return;
+    const int64_t t_end = (t_start + TILE < n) ? t_start + TILE : n;
+    const bool last_tile = (t_end >= n);
+    constexpr int CH = 4;
+#pragma unroll 1
+    for (int rr = 0; rr < RPW; ++rr) {
+        const int local = warp * RPW + rr;
+        const int64_t row = t_start + local;
+        int keep = 0;
+        if (row < n) {
+            const char* u = a.U + row * a.ldU_b;
+            const char* h = a.H + row * a.ldH_b;
+            char* o = a.x_full + (int64_t)a.tok_in[row] * a.ldx_b;
+            float su = 0.f, sh = 0.f;
+            for (int base = 0; base < a.nvec; base += 32 * CH) {
+                uint4 x[CH], y[CH];
+#pragma unroll
+                for (int k = 0; k < CH; ++k) {
+                    const int v = base + k * 32 + lane;
+                    if (v < a.nvec) { x[k] = ld_nc_v4(u + ((int64_t)v << 4)); y[k] = ld_nc_v4(h + ((int64_t)v << 4)); }
+                }
+#pragma unroll
+                for (int k = 0; k < CH; ++k) {
+                    const int v = base + k * 32 + lane;
+                    if (v < a.nvec) {
+                        su += sumsq_vec<BF16>(x[k]);
+                        sh += sumsq_vec<BF16>(y[k]);
+                        st_v4(o + ((int64_t)v << 4), add_vec<BF16>(x[k], y[k]));
+                    }
+                }
+            }
+            su = warp_sum(su);
+            sh = warp_sum(sh);
+            const float num = sqrtf(su);
+            const float r = (a.mode == DASH_NORM_ABS) ? num : num / fmaxf(sqrtf(sh), a.eps);
+            const int s = find_seq(a.cu_in, a.S, (int)row);
+            const int lp = (int)row - a.cu_in[s], len = a.cu_in[s + 1] - a.cu_in[s];
+            const bool prot = (lp < a.keep_first) || (lp >= len - a.keep_last);
+            keep = (prot || !(r < a.tau)) ? 1 : 0;
+            if (lane == 0) { a.r_out[row] = r; a.mask_out[row] = (uint8_t)keep; }
+        }
+        if (lane == 0) s_keep[local] = keep;
+    }
+    __syncthreads();                                    // also orders this CTA's x_full rows before the copies below
+    if (warp == 0) {
+        const int my = s_keep[lane];
+        const unsigned int bal = __ballot_sync(0xffffffffu, my);
+        const int agg = __popc(bal);
+        int base = 0;
+        if (tile == 0) {
+            if (lane == 0) st_state(&a.tile_state[0], kFlagPrefix | (unsigned int)agg);
+        } else {
+            if (lane == 0) st_state(&a.tile_state[tile], kFlagAgg | (unsigned int)agg);
+            int look = tile - 1;
+            bool done = false, timed_out = false;
+            while (!done) {
+                const int j = look - lane;
+                unsigned long long st = kFlagPrefix;
+                uint32_t spins = 0;
+                if (j >= 0) {
+                    st = ld_state(&a.tile_state[j]);
+                    while ((st >> 32) == 0) {
+                        if (++spins > kSpinLimit) { timed_out = true; break; }
+                        __nanosleep(32);
+                        st = ld_state(&a.tile_state[j]);
+                    }
+                }
+                if (__any_sync(0xffffffffu, timed_out)) { timed_out = true; break; }
+                const unsigned int has_prefix = __ballot_sync(0xffffffffu, (st >> 32) == 2);
+                const int first = has_prefix ? (__ffs(has_prefix) - 1) : 32;
+                int v = (lane <= first) ? (int)(unsigned int)(st & 0xffffffffu) : 0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                base += v;
+                if (has_prefix) done = true; else look -= 32;
+            }
+            if (timed_out) { if (lane == 0) atomicExch(a.status, DASH_ERR_TIMEOUT); base = 0; }
+            if (lane == 0) st_state(&a.tile_state[tile], kFlagPrefix | (unsigned int)(base + agg));
+        }
+        if (my) {
+            const int k = __popc(bal & ((1u << lane) - 1u));
+            const int t = (int)t_start + lane;
+            s_src[k] = t;
+            a.tok_next[base + k] = a.tok_in[t];
+            a.pos_next[base + k] = a.pos_in[t];
+        }
+        if (lane == 0) { s_base = base; s_count = agg; s_ballot = bal; }
+    }
+    __syncthreads();
+    const int base = s_base, count = s_count;
+    const unsigned int bal = s_ballot;
+    for (int s = threadIdx.x; s <= a.S; s += blockDim.x) {
+        int64_t c = a.cu_in[s];
+        if (c > n) c = n;
+        bool mine = (c >= t_start && c < t_start + TILE && c < t_end) || (last_tile && c == t_end);
+        if (tile == 0 && n == 0) mine = true;
+        if (mine) {
+            const int p = (int)(c - t_start);
+            int v = base;
+            if (p >= TILE || c >= t_end) v += count;
+            else v += __popc(bal & ((1u << p) - 1u));
+            a.cu_next[s] = v;
+            if (s == a.S && a.n_next) *a.n_next = v;
+        }
+    }
+    // copy the tile's active rows x_full[tok] -> H_next[base + k], 4 KB pieces dealt to the warps
+    const int64_t rb = (int64_t)a.nvec << 4;
+    const int pieces = (int)((rb + kPieceBytes - 1) / kPieceBytes);
+    const int items = count * pieces;
+    for (int it = warp; it < items; it += NWARPS) {
+        const int k = it / pieces, pc = it - k * pieces;
+        const int64_t off = (int64_t)pc * kPieceBytes;
+        const int nv = (int)(((rb - off < kPieceBytes) ? rb - off : kPieceBytes) >> 4);
+        const char* src = a.x_full + (int64_t)a.tok_in[s_src[k]] * a.ldx_b + off;
+        char* dst = a.H_next + (int64_t)(base + k) * a.ldn_b + off;
+        uint4 r[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) { const int v = q * 32 + lane; if (v < nv) r[q] = ld_cg_v4(src + ((int64_t)v << 4)); }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) { const int v = q * 32 + lane; if (v < nv) st_v4(dst + ((int64_t)v << 4), r[q]); }
+    }
+}
+
 static int rows_grid(int64_t n, int wpb) {
     int64_t blocks = (n + wpb - 1) / wpb;
     int64_t cap = (int64_t)sm_count() * 8;     // 8 CTAs of 256 threads fill an SM
@@ -612,5 +772,29 @@ extern "C" int dash_compact_static(const uint8_t* mask, int64_t n, const int32_t
 
 namespace dash {
 size_t select_ws_bytes(int64_t, int) { return 256; }
+
+// Fused tail of the block step (see delta_tail_kernel).  Preconditions checked by the caller: threshold rule, every row
+// scattered, 16-byte aligned rows.  ws: the compaction workspace (ticket + one state word per 32-token tile).
+int launch_delta_tail(const void* U, const void* H, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
+                      int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
+                      void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
+                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st) {
+    const int es = dt == DASH_BF16 ? 2 : 4;
+    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < compact_ws_bytes(n)) return DASH_ERR_WORKSPACE;
+    const int tiles = (int)((n + 31) / 32) > 0 ? (int)((n + 31) / 32) : 1;
+    DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)tiles * 8, st));
+    TailArgs a;
+    a.U = (const char*)U; a.H = (const char*)H; a.ldU_b = a.ldH_b = (int64_t)d * es; a.nvec = d * es / 16; a.mode = (int)mode; a.eps = eps;
+    a.tau = tau; a.keep_first = keep_first; a.keep_last = keep_last; a.cu_in = cu_in; a.S = S; a.tok_in = tok_in; a.pos_in = pos_in;
+    a.x_full = (char*)x_full; a.ldx_b = (int64_t)d * es; a.H_next = (char*)H_next; a.ldn_b = (int64_t)d * es;
+    a.r_out = r_out; a.mask_out = mask_out; a.tok_next = tok_next; a.pos_next = pos_next; a.cu_next = cu_next; a.n_next = n_next;
+    a.ticket = (unsigned int*)ws; a.tile_state = (unsigned long long*)((char*)ws + 256);
+    a.status = status_word_ptr();
+    if (!a.status) return DASH_ERR_CUDA;
+    if (dt == DASH_BF16) delta_tail_kernel<true><<<tiles, kCompactThreads, 0, st>>>(a, n);
+    else delta_tail_kernel<false><<<tiles, kCompactThreads, 0, st>>>(a, n);
+    DASH_CUDA_TRY(cudaGetLastError());
+    return DASH_OK;
+}
 size_t compact_ws_bytes_pub(int64_t n) { return compact_ws_bytes(n); }
 }  // namespace dash

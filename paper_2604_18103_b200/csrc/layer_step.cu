@@ -165,6 +165,11 @@ static int gemm_rowmajor(dash_dtype dt, const void* A, int64_t lda, const void* 
     return rc;
 }
 
+int launch_delta_tail(const void* U, const void* H, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
+                      int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
+                      void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
+                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st);
+
 static int rows_grid8(int64_t n) {
     int64_t blocks = (n + 7) / 8, cap = (int64_t)sm_count() * 8;
     if (blocks > cap) blocks = cap;
@@ -260,6 +265,12 @@ extern "C" int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, cons
         if (rc != DASH_OK) return rc;
         // U = O Wo  (pre-residual attention output, Eq. 1)
         if ((rc = gemm_rowmajor(cfg->dt, O, (int64_t)Hq * D, cfg->Wo, d, U, d, n, d, (int64_t)Hq * D, lt_ws, st)) != DASH_OK) return rc;
+        if (cfg->sel_mode == DASH_SEL_THRESHOLD && cfg->scatter_which == 2) {
+            // r, H~ = H + U, the halting rule, the scatter of H~ and the compaction of the rows that stay, in one pass
+            return launch_delta_tail(U, H_in, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau, cfg->keep_first, cfg->keep_last,
+                                     cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out, tok_index_next, pos_next,
+                                     cu_next, n_next_dev, compact_ws, compact_bytes, st);
+        }
         // r, H~ = H + U, and (threshold mode) the halting rule in the same pass
         dash_threshold ft = {cfg->tau, cfg->keep_first, cfg->keep_last, cu_in, S, mask_out};
         rc = dash_delta_norm(U, H_in, n, d, d, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, r_out, Ht, d, nullptr,

@@ -60,7 +60,7 @@ def test_config2_block_step_full_size():
     # ~0.5-1 % per element, and the maximum over d = 3584 elements of a row sits 4.2 sigma above that.  Bar for this
     # intermediate: 6e-2 of the row RMS; the state outputs below (H~, r, mask, x_full) meet the 2e-2 bar.
     assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype)[rows].float().cpu().numpy(), ref["U"], "U (sampled rows)", tol=6e-2)
-    Ht = bufs.view(bufs.lay.Ht, T, sh.d, sh.dtype)
+    Ht = x_full                                         # H~ of every entry token (tok is the identity): written by the fused tail pass
     assert_close_rms(Ht[rows].float().cpu().numpy(), ref["Ht"], "H~ (sampled rows)")
     r_gpu, mask = bufs.r.cpu().numpy(), bufs.mask.cpu().numpy()
     assert np.array_equal(r_gpu, r0)                                    # deterministic
@@ -75,7 +75,6 @@ def test_config2_block_step_full_size():
     assert torch.equal(bufs.H_next[:k].cpu(), Ht.cpu()[idx])            # gather is bit-exact
     assert np.array_equal(bufs.tok_next[:k].cpu().numpy(), idx) and np.array_equal(bufs.pos_next[:k].cpu().numpy(), idx)
     assert bufs.cu_next.cpu().tolist() == [0, k]
-    assert torch.equal(x_full.cpu(), Ht.cpu())
 
 
 def test_config3_cascade_full_size_properties():
@@ -108,9 +107,9 @@ def test_config3_cascade_full_size_properties():
         assert k == Ks[l], (l, k, Ks[l])                        # n' sequence = floor(f_l T)
         if l == 0:
             assert_close_rms(out.view(out.lay.U, T, sh.d, sh.dtype)[rows].float().cpu().numpy(), ref["U"], "layer-1 U (sampled rows)", tol=6e-2)
-            assert_close_rms(out.view(out.lay.Ht, T, sh.d, sh.dtype)[rows].float().cpu().numpy(), ref["Ht"], "layer-1 H~ (sampled rows)")
+            assert_close_rms(x_full[rows].float().cpu().numpy(), ref["Ht"], "layer-1 H~ (sampled rows)")
             assert np.max(np.abs(out.r.cpu().numpy()[rows] - ref["r"]) / ref["r"]) < 2e-2
-            assert torch.equal(out.H_next[:k], out.view(out.lay.Ht, T, sh.d, sh.dtype)[:k])   # keep-all: identity path
+            assert torch.equal(out.H_next[:k], x_full[:k])      # keep-all: identity path
         tok_in = tok[:n_l].cpu().numpy()
         mask = out.mask[:n_l].cpu().numpy()
         tok_out = out.tok_next[:k].cpu().numpy()

@@ -85,7 +85,9 @@ def test_layer_step_matches_oracle(cfg):
     assert_close_rms(bufs.view(bufs.lay.O, T, sh.Hq * sh.D, sh.dtype).float().cpu().numpy(), ref["O"].reshape(T, -1), "attention O",
                      atol=(2.0 ** (math.floor(math.log2(float(np.abs(ref["V"]).max()))) - 8)) if sh.dtype == torch.bfloat16 else 0.0)
     assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype).float().cpu().numpy(), ref["U"], "U")
-    assert_close_rms(bufs.view(bufs.lay.Ht, T, sh.d, sh.dtype).float().cpu().numpy(), ref["Ht"], "H~")
+    # H~ of every entry token reaches x_full (threshold rule: score, residual, scatter and compaction run as one pass,
+    # which writes H~ there and nowhere else); tok is the identity here
+    assert_close_rms(x_full.float().cpu().numpy(), ref["Ht"], "H~ (x_full)")
     r_gpu = bufs.r.cpu().numpy()
     assert np.max(np.abs(r_gpu - ref["r"]) / ref["r"]) < 2e-2
     mask = bufs.mask.cpu().numpy()
@@ -94,13 +96,11 @@ def test_layer_step_matches_oracle(cfg):
     idx = np.flatnonzero(mask)
     k = int(bufs.n_next.item())
     assert k == idx.size and abs(k - K) <= flips
-    Ht_gpu = bufs.view(bufs.lay.Ht, T, sh.d, sh.dtype)
-    assert torch.equal(bufs.H_next[:k].cpu(), Ht_gpu.cpu()[idx])
+    assert torch.equal(bufs.H_next[:k].cpu(), x_full.cpu()[idx])         # gathered rows are bit-exact copies
     assert np.array_equal(bufs.tok_next[:k].cpu().numpy(), idx)
     assert np.array_equal(bufs.pos_next[:k].cpu().numpy(), pos.numpy()[idx])
     cu_ref = np.concatenate([[0], np.cumsum([mask[int(w.cu[s]):int(w.cu[s + 1])].sum() for s in range(S)])])
     assert np.array_equal(bufs.cu_next.cpu().numpy(), cu_ref)
-    assert torch.equal(x_full.cpu(), Ht_gpu.cpu())                       # scatter of every entry token
     if flips == 0:                                                       # then everything equals the oracle's own compaction
         assert np.array_equal(idx, ref["idx"]) and np.array_equal(cu_ref, ref["cu_out"])
         assert_close_rms(bufs.H_next[:k].float().cpu().numpy(), ref["rows"][0], "H_next")
