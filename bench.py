@@ -42,7 +42,7 @@ UNIT = "tokens/s"
 L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch (ncu, profiles/attention_kernel_cfg2_8192.md); null where
 # no capture of the current kernel exists
-ATTN_TRAFFIC = {"cfg2": 93.47e6}
+ATTN_TRAFFIC = {"cfg2": 94.74e6}
 
 
 def rank_seed(base: int, rank: int) -> int:
