@@ -215,6 +215,21 @@ def test_attention_qwen_heads_sampled_rows():
     _attention_case(lengths, 28, 4, 128, torch.bfloat16, 6, rows=rows.numpy())
 
 
+def test_attention_many_short_sequences_some_empty():
+    # 150 sequences of 0..200 tokens: more work items than persistent CTAs, most query tiles ragged
+    g = torch.Generator().manual_seed(11)
+    lengths = torch.randint(0, 201, (150,), generator=g).tolist()
+    lengths[7] = lengths[80] = 0
+    _attention_case(lengths, 4, 2, 128, torch.bfloat16, 11, pad=3)
+
+
+def test_attention_one_long_sequence_more_than_1024_query_tiles():
+    # 1031 query tiles: the plan of work items is built in more than one pass over the tile levels
+    n = 1031 * 128 - 5
+    rows = wl.sample_rows(wl.cu_from_lengths([n]), 48, seed=12)
+    _attention_case([n], 1, 1, 64, torch.bfloat16, 12, rows=rows.numpy())
+
+
 def test_attention_closed_forms_on_device():
     # V constant -> O constant; Q = 0 -> prefix mean (uniform weights)
     n, Hq, Hkv, D = 400, 2, 1, 128

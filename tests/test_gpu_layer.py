@@ -185,3 +185,47 @@ def test_cascade_small_matches_oracle():
     got = x_full.float().cpu().numpy()[same]
     assert_close_rms(got, x_o[same], "x_full after the cascade", tol=2e-2 * math.sqrt(8))
     assert math.sqrt(float(np.mean((got - x_o[same]) ** 2))) < 1e-2
+
+
+def test_layer_step_rows_beyond_the_packed_end_and_protected_tokens():
+    """Buffers allocated for more rows than the batch holds (the true count lives in cu_seqlens[S] on the device),
+    poisoned rows past the end, permuted rows in the full-length buffer, protected prefix/suffix under the threshold rule."""
+    w = wl.config2(T=700, seed=25, shape=wl.MINI)
+    w.cu = wl.cu_from_lengths([257, 0, 443])
+    sh, T, S = w.shape, w.T, w.S
+    H, W = w.tensors["H"], w.weights[0]
+    pos = wl.positions(w.cu)
+    kf, kl, pad = 5, 3, 77
+    ref0 = oc.layer_step(H, W, w.cu, pos, sh, tau=0.0)
+    tau = oc.kth_largest(ref0["r"], T // 2)
+    ref = oc.layer_step(H, W, w.cu, pos, sh, tau=tau, keep_first=kf, keep_last=kl)
+    g = torch.Generator().manual_seed(3)
+    perm = torch.randperm(T + pad, generator=g)[:T].to(torch.int32)          # rows of the tokens in the full-length buffer
+    Hp = torch.cat([H, torch.full((pad, sh.d), float("nan"), dtype=sh.dtype)])
+    tokp = torch.cat([perm, torch.full((pad,), 0, dtype=torch.int32)])
+    posp = torch.cat([pos, torch.zeros(pad, dtype=torch.int32)])
+    layer = dash.Layer(sh, W, DEV, tau=tau, keep_first=kf, keep_last=kl)
+    bufs = StepBuffers(layer, T + pad, S, T + pad, sh.dtype)
+    x_full = torch.full((T + pad, sh.d), 9.0, dtype=sh.dtype, device=DEV)
+    run_step(layer, Hp.to(DEV), tokp.to(DEV), posp.to(DEV), w.cu.to(DEV), 443, x_full, bufs)
+    mask = bufs.mask[:T].cpu().numpy()
+    r_gpu = bufs.r[:T].cpu().numpy()
+    assert np.max(np.abs(r_gpu - ref["r"]) / ref["r"]) < 2e-2
+    flips, _ = check_mask(mask, r_gpu, ref["r"], tau, w.cu, kf, kl)
+    for s in range(S):
+        a, b = int(w.cu[s]), int(w.cu[s + 1])
+        assert mask[a:min(a + kf, b)].all() and mask[max(b - kl, a):b].all()
+    k = int(bufs.n_next.item())
+    idx = np.flatnonzero(mask)
+    assert k == idx.size
+    xf = x_full.cpu()
+    assert_close_rms(xf[perm.long()].float().numpy(), ref["Ht"], "H~ at the tokens' rows of x_full")
+    untouched = np.setdiff1d(np.arange(T + pad), perm.numpy())
+    assert (xf[untouched] == 9.0).all()                                      # nothing written for rows past the packed end
+    assert torch.equal(bufs.H_next[:k].cpu(), xf[perm.long()][idx])
+    assert np.array_equal(bufs.tok_next[:k].cpu().numpy(), perm.numpy()[idx])
+    assert np.array_equal(bufs.pos_next[:k].cpu().numpy(), pos.numpy()[idx])
+    cu_ref = np.concatenate([[0], np.cumsum([mask[int(w.cu[s]):int(w.cu[s + 1])].sum() for s in range(S)])])
+    assert np.array_equal(bufs.cu_next.cpu().numpy(), cu_ref)
+    if flips == 0:
+        assert np.array_equal(mask, ref["mask"])
