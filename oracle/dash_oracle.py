@@ -317,6 +317,34 @@ def layer_step(H, weights: Dict[str, object], cu, pos, shape, norm_mode: int = R
     return out
 
 
+def ffn_swiglu(X, Wg, Wu, Wd) -> np.ndarray:
+    """FFN of Alg. 1, read as the gated feed-forward of the Qwen2.5 backbones:
+    FFN(x) = (silu(x Wg) * (x Wu)) Wd with silu(z) = z / (1 + exp(-z))."""
+    X = f64(X)
+    g = X @ f64(Wg)
+    u = X @ f64(Wu)
+    return ((g / (1.0 + np.exp(-g))) * u) @ f64(Wd)
+
+
+def block_step(H, weights: Dict[str, object], cu, pos, shape, norm_mode: int = REL,
+               sel_mode: int = THRESHOLD, tau: float = 0.0, keep_counts=None,
+               keep_first: int = 0, keep_last: int = 0, eps: float = 1e-12,
+               attn_rows=None) -> Dict[str, object]:
+    """One whole block of Alg. 1 on the packed active tokens: U = Attn(LN(H)); H~ = H + U;
+    H' = H~ + FFN(LN(H~)); the score is taken from U, the selection from the score; the tokens that
+    stay carry H' into the next block, and H' is also the last updated value of the tokens that halt
+    here (Sec. 3.4).  `weights` holds the attention weights of layer_step plus Wg, Wu, Wd, rms2_w.
+    With attn_rows given only those rows are evaluated (no selection)."""
+    out = layer_step(H, weights, cu, pos, shape, norm_mode, sel_mode, tau, keep_counts, keep_first, keep_last, eps, attn_rows)
+    Hn2 = rmsnorm(out["Ht"], weights["rms2_w"], shape.rms_eps)
+    out["F"] = ffn_swiglu(Hn2, weights["Wg"], weights["Wu"], weights["Wd"])
+    out["H1"] = out["Ht"] + out["F"]
+    if attn_rows is not None:
+        return out
+    out.update(compact(out["mask"], cu, rows=[out["H1"]], pos_in=pos))
+    return out
+
+
 def kth_largest(r, k: int) -> float:
     """The k-th largest score (k >= 1): with tau set to it and the rule
     "halt iff r < tau", exactly k tokens stay when there are no ties."""

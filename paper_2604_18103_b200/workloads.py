@@ -32,16 +32,17 @@ class LayerShape:
     rope_base: float
     dtype: torch.dtype
     rms_eps: float = 1e-6
+    m: int = 0      # feed-forward width (0: the block is used without its FFN)
 
     @property
     def G(self) -> int:
         return self.Hq // self.Hkv
 
 
-QWEN = LayerShape(d=3584, Hq=28, Hkv=4, D=128, rope_base=1.0e6, dtype=torch.bfloat16)
-TINY = LayerShape(d=256, Hq=4, Hkv=4, D=64, rope_base=1.0e4, dtype=torch.float32)
+QWEN = LayerShape(d=3584, Hq=28, Hkv=4, D=128, rope_base=1.0e6, dtype=torch.bfloat16, m=18944)
+TINY = LayerShape(d=256, Hq=4, Hkv=4, D=64, rope_base=1.0e4, dtype=torch.float32, m=512)
 # Qwen-like GQA shape small enough for full CPU checks of every row
-MINI = LayerShape(d=512, Hq=8, Hkv=2, D=128, rope_base=1.0e6, dtype=torch.bfloat16)
+MINI = LayerShape(d=512, Hq=8, Hkv=2, D=128, rope_base=1.0e6, dtype=torch.bfloat16, m=1024)
 
 # active fraction after each layer of the cascaded workload (config 3)
 CASCADE_FRACTIONS = (1.0, 0.9, 0.8, 0.7, 0.6, 0.5, 0.4, 0.35)
@@ -77,6 +78,17 @@ def layer_weights(shape: LayerShape, seed: int, layer: int = 0) -> Dict[str, tor
         "Wv": _randn((shape.d, shape.Hkv * shape.D), seed, s + 3, 0.02, shape.dtype),
         "Wo": _randn((shape.Hq * shape.D, shape.d), seed, s + 4, 0.02, shape.dtype),
         "rms_w": torch.ones(shape.d, dtype=shape.dtype),
+    }
+
+
+def ffn_weights(shape: LayerShape, seed: int, layer: int = 0) -> Dict[str, torch.Tensor]:
+    """Gated feed-forward weights of width shape.m: Wg, Wu [d, m], Wd [m, d] ~ N(0, 0.02^2), second RMSNorm weight = 1."""
+    s = 100 + 10 * layer
+    return {
+        "Wg": _randn((shape.d, shape.m), seed, s + 5, 0.02, shape.dtype),
+        "Wu": _randn((shape.d, shape.m), seed, s + 6, 0.02, shape.dtype),
+        "Wd": _randn((shape.m, shape.d), seed, s + 7, 0.02, shape.dtype),
+        "rms2_w": torch.ones(shape.d, dtype=shape.dtype),
     }
 
 

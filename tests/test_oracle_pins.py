@@ -344,6 +344,40 @@ def test_layer_step_against_torch_restatement_and_rho0():
     assert np.allclose(res3["U"], res["U"][[0, 100, 191]], rtol=1e-12, atol=1e-14)
 
 
+def test_block_step_ffn_against_torch_restatement_and_closed_forms():
+    w = wl.config2(T=160, seed=12, shape=wl.MINI)
+    sh = w.shape
+    W = dict(w.weights[0]); W.update(wl.ffn_weights(sh, 12))
+    H, pos = w.tensors["H"], wl.positions(w.cu)
+    K = oc.keep_count(160, 0.5)
+    base = oc.layer_step(H, W, w.cu, pos, sh, tau=0.0)
+    tau = oc.kth_largest(base["r"], K)
+    res = oc.block_step(H, W, w.cu, pos, sh, tau=tau)
+    # independent restatement with library routines (torch fp64 matmul, silu, rms norm by hand)
+    _, Ht = _torch_layer(H, W, pos, sh)
+    x = Ht / torch.sqrt(Ht.pow(2).mean(dim=1, keepdim=True) + sh.rms_eps) * W["rms2_w"].double()
+    F = (torch.nn.functional.silu(x @ W["Wg"].double()) * (x @ W["Wu"].double())) @ W["Wd"].double()
+    assert np.allclose(res["F"], F.numpy(), rtol=1e-9, atol=1e-12)
+    assert np.allclose(res["H1"], (Ht + F).numpy(), rtol=1e-9, atol=1e-12)
+    # the FFN changes neither the score nor the selection (both come from U), only what is carried on
+    assert np.array_equal(res["r"], base["r"]) and int(res["mask"].sum()) == K
+    assert np.array_equal(res["rows"][0], res["H1"][res["mask"].astype(bool)])
+    # closed forms: a zero down projection or a zero gate leaves H~ unchanged; silu(z) -> z for large z
+    for zero in ("Wd", "Wg"):
+        Wz = dict(W); Wz[zero] = torch.zeros_like(W[zero])
+        rz = oc.block_step(H, Wz, w.cu, pos, sh, tau=tau)
+        assert np.array_equal(rz["H1"], rz["Ht"])
+    X = np.full((1, 2), 40.0)
+    eye = np.eye(2)
+    assert np.allclose(oc.ffn_swiglu(X, eye, eye, eye), X * X, rtol=1e-12)       # silu(40) = 40 to 1e-17
+    assert np.allclose(oc.ffn_swiglu(-X, eye, eye, eye), 0.0, atol=1e-12)        # silu(-40) ~ -1.7e-16
+    assert abs(oc.ffn_swiglu(np.array([[1.0]]), np.array([[1.0]]), np.array([[2.0]]), np.array([[3.0]]))[0, 0]
+               - (1.0 / (1.0 + math.exp(-1.0))) * 2.0 * 3.0) < 1e-15
+    # row-sampled evaluation equals the full one on those rows
+    r3 = oc.block_step(H, W, w.cu, pos, sh, attn_rows=[0, 77, 159])
+    assert np.allclose(r3["H1"], res["H1"][[0, 77, 159]], rtol=1e-12, atol=1e-13)
+
+
 def test_workload_recipes_have_stated_structure():
     w4 = wl.config4(T=4096, seed=3, shape=wl.MINI)
     r = oc.delta_norm(w4.tensors["U"], w4.tensors["H"])
