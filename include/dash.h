@@ -221,6 +221,32 @@ int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, const int32_t* 
                     int32_t* cu_next, int32_t* n_next_dev, float* r_out, uint8_t* mask_out,
                     void* ws, size_t ws_bytes, void* stream);
 
+/* ---- the whole block of Alg. 1, feed-forward included ----------------------
+ * H' = H~ + FFN(LN(H~)) with H~ = H + U as above; the score and the selection still
+ * come from U.  FFN is the gated feed-forward of the Qwen2.5 backbones:
+ * FFN(x) = (silu(x Wg) * (x Wu)) Wd.  H' of every entering token is written to x_full
+ * (attn.scatter_which must be 2: H' is also the last updated value of the tokens that
+ * halt here, Sec. 3.4), H' of the tokens that stay to H_next.  Projections are library
+ * GEMMs; everything else runs in this library's kernels. */
+typedef struct {
+    dash_layer_cfg attn;
+    int          m;                /* feed-forward width, multiple of 8 */
+    const void*  Wgu;              /* [d, 2 m]: columns = Wg | Wu */
+    const void*  Wd;               /* [m, d] */
+    const void*  rms2_weight;      /* [d]: weight of the norm in front of the FFN (attn.rms_eps is used) */
+} dash_block_cfg;
+typedef struct {
+    dash_layer_ws_layout attn;
+    size_t GU, ACT, F, total;      /* gate | up [n, 2m], activation [n, m], FFN output [n, d] */
+} dash_block_ws_layout;
+int dash_block_workspace(const dash_block_cfg* cfg, int64_t n, int S, dash_block_ws_layout* out);
+/* Arguments as dash_layer_step. */
+int dash_block_step(const dash_block_cfg* cfg, const void* H_in, const int32_t* tok_index_in,
+                    const int32_t* pos_in, const int32_t* cu_in, int S, int64_t n, int64_t max_seqlen,
+                    void* x_full, void* H_next, int32_t* tok_index_next, int32_t* pos_next,
+                    int32_t* cu_next, int32_t* n_next_dev, float* r_out, uint8_t* mask_out,
+                    void* ws, size_t ws_bytes, void* stream);
+
 /* ---- workspace sizes ------------------------------------------------------ */
 typedef enum { DASH_WS_SELECT = 0, DASH_WS_COMPACT = 1, DASH_WS_ATTENTION = 2 } dash_ws_op;
 /* n: rows allocated; S: sequences; Hq, Hkv, D, dt only matter for attention. */

@@ -437,6 +437,7 @@ __device__ __forceinline__ uint4 ld_cg_v4(const void* p) {
 
 struct TailArgs {
     const char* U; const char* H; int64_t ldU_b, ldH_b; int nvec; int mode; float eps;
+    const uint8_t* mask_in;       // non-null: keep decisions are given (r and the mask are not formed), U is any update to add to H
     float tau; int keep_first, keep_last; const int32_t* cu_in; int S;
     const int32_t* tok_in; const int32_t* pos_in;
     char* x_full; int64_t ldx_b; char* H_next; int64_t ldn_b;
@@ -490,15 +491,19 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
                     }
                 }
             }
-            su = warp_sum(su);
-            sh = warp_sum(sh);
-            const float num = sqrtf(su);
-            const float r = (a.mode == DASH_NORM_ABS) ? num : num / fmaxf(sqrtf(sh), a.eps);
-            const int s = find_seq(a.cu_in, a.S, (int)row);
-            const int lp = (int)row - a.cu_in[s], len = a.cu_in[s + 1] - a.cu_in[s];
-            const bool prot = (lp < a.keep_first) || (lp >= len - a.keep_last);
-            keep = (prot || !(r < a.tau)) ? 1 : 0;
-            if (lane == 0) { a.r_out[row] = r; a.mask_out[row] = (uint8_t)keep; }
+            if (a.mask_in) {
+                keep = a.mask_in[row] != 0;
+            } else {
+                su = warp_sum(su);
+                sh = warp_sum(sh);
+                const float num = sqrtf(su);
+                const float r = (a.mode == DASH_NORM_ABS) ? num : num / fmaxf(sqrtf(sh), a.eps);
+                const int s = find_seq(a.cu_in, a.S, (int)row);
+                const int lp = (int)row - a.cu_in[s], len = a.cu_in[s + 1] - a.cu_in[s];
+                const bool prot = (lp < a.keep_first) || (lp >= len - a.keep_last);
+                keep = (prot || !(r < a.tau)) ? 1 : 0;
+                if (lane == 0) { a.r_out[row] = r; a.mask_out[row] = (uint8_t)keep; }
+            }
         }
         if (lane == 0) s_keep[local] = keep;
     }
@@ -775,7 +780,7 @@ size_t select_ws_bytes(int64_t, int) { return 256; }
 
 // Fused tail of the block step (see delta_tail_kernel).  Preconditions checked by the caller: threshold rule, every row
 // scattered, 16-byte aligned rows.  ws: the compaction workspace (ticket + one state word per 32-token tile).
-int launch_delta_tail(const void* U, const void* H, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
+int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
                       int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st) {
@@ -784,6 +789,7 @@ int launch_delta_tail(const void* U, const void* H, int64_t n, int d, dash_dtype
     const int tiles = (int)((n + 31) / 32) > 0 ? (int)((n + 31) / 32) : 1;
     DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)tiles * 8, st));
     TailArgs a;
+    a.mask_in = mask_in;
     a.U = (const char*)U; a.H = (const char*)H; a.ldU_b = a.ldH_b = (int64_t)d * es; a.nvec = d * es / 16; a.mode = (int)mode; a.eps = eps;
     a.tau = tau; a.keep_first = keep_first; a.keep_last = keep_last; a.cu_in = cu_in; a.S = S; a.tok_in = tok_in; a.pos_in = pos_in;
     a.x_full = (char*)x_full; a.ldx_b = (int64_t)d * es; a.H_next = (char*)H_next; a.ldn_b = (int64_t)d * es;

@@ -165,7 +165,7 @@ static int gemm_rowmajor(dash_dtype dt, const void* A, int64_t lda, const void* 
     return rc;
 }
 
-int launch_delta_tail(const void* U, const void* H, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
+int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
                       int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st);
@@ -174,6 +174,38 @@ static int rows_grid8(int64_t n) {
     int64_t blocks = (n + 7) / 8, cap = (int64_t)sm_count() * 8;
     if (blocks > cap) blocks = cap;
     return (int)(blocks < 1 ? 1 : blocks);
+}
+
+
+// act[t, j] = silu(GU[t, j]) * GU[t, m + j]   (gated feed-forward; silu(z) = z / (1 + exp(-z))), 8 (bf16) or 4 (fp32) columns per thread
+template <bool BF16>
+__global__ void __launch_bounds__(256)
+swiglu_kernel(const char* __restrict__ GU, int64_t ldgu_b, char* __restrict__ ACT, int64_t lda_b, int64_t n, int m,
+              const int32_t* __restrict__ n_dev) {
+    constexpr int ES = BF16 ? 2 : 4, EPV = 16 / ES;
+    if (n_dev) { int64_t nd = *n_dev; if (nd < n) n = nd; }
+    const int vpr = m / EPV;                              // 16-byte vectors per output row
+    const int64_t total = n * vpr;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t t = i / vpr;
+        const int v = (int)(i - t * vpr);
+        const uint4 g = ld_nc_v4(GU + t * ldgu_b + ((int64_t)v << 4));
+        const uint4 u = ld_nc_v4(GU + t * ldgu_b + (int64_t)m * ES + ((int64_t)v << 4));
+        auto act = [](float a, float b) { return a / (1.0f + __expf(-a)) * b; };
+        uint4 o;
+        if (BF16) {
+            o.x = pack_bf16(act(bf16lo(g.x), bf16lo(u.x)), act(bf16hi(g.x), bf16hi(u.x)));
+            o.y = pack_bf16(act(bf16lo(g.y), bf16lo(u.y)), act(bf16hi(g.y), bf16hi(u.y)));
+            o.z = pack_bf16(act(bf16lo(g.z), bf16lo(u.z)), act(bf16hi(g.z), bf16hi(u.z)));
+            o.w = pack_bf16(act(bf16lo(g.w), bf16lo(u.w)), act(bf16hi(g.w), bf16hi(u.w)));
+        } else {
+            o.x = __float_as_uint(act(__uint_as_float(g.x), __uint_as_float(u.x)));
+            o.y = __float_as_uint(act(__uint_as_float(g.y), __uint_as_float(u.y)));
+            o.z = __float_as_uint(act(__uint_as_float(g.z), __uint_as_float(u.z)));
+            o.w = __float_as_uint(act(__uint_as_float(g.w), __uint_as_float(u.w)));
+        }
+        st_v4(ACT + t * lda_b + ((int64_t)v << 4), o);
+    }
 }
 
 static bool cfg_ok(const dash_layer_cfg* c) {
@@ -211,6 +243,91 @@ extern "C" int dash_layer_workspace(const dash_layer_cfg* cfg, int64_t n, int S,
     return DASH_OK;
 }
 
+namespace dash {
+
+struct StepWs {
+    dash_layer_ws_layout L;
+    char *Hn, *QKV, *O, *U, *Ht, *lt_ws, *compact_ws, *attn_ws;
+    size_t compact_bytes, attn_bytes;
+};
+
+static int carve_ws(const dash_layer_cfg* cfg, int64_t n, int S, void* ws, StepWs* out) {
+    int rc = dash_layer_workspace(cfg, n, S, &out->L);
+    if (rc != DASH_OK) return rc;
+    char* w = (char*)ws;
+    out->Hn = w + out->L.Hn; out->QKV = w + out->L.QKV; out->O = w + out->L.O; out->U = w + out->L.U; out->Ht = w + out->L.Ht;
+    out->lt_ws = w + out->L.scratch;
+    out->compact_ws = out->lt_ws + kLtWorkspace;
+    out->compact_bytes = align_up(dash_workspace_bytes(DASH_WS_COMPACT, n, S, 0, 0, 0, cfg->dt), 256);
+    out->attn_ws = out->compact_ws + out->compact_bytes;
+    out->attn_bytes = dash_workspace_bytes(DASH_WS_ATTENTION, n, S, cfg->Hq, cfg->Hkv, cfg->D, cfg->dt);
+    return DASH_OK;
+}
+
+static int launch_rmsnorm(dash_dtype dt, const void* X, const void* weight, void* Y, int64_t n, int d, float eps, const int32_t* n_dev,
+                          cudaStream_t st) {
+    const int es = dt == DASH_BF16 ? 2 : 4, nvec = d * es / 16;
+    if (dt == DASH_BF16) rmsnorm_kernel<true><<<rows_grid8(n), 256, 0, st>>>((const char*)X, (int64_t)d * es, (const char*)weight, (char*)Y, (int64_t)d * es, n, nvec, 1.f / d, eps, n_dev);
+    else rmsnorm_kernel<false><<<rows_grid8(n), 256, 0, st>>>((const char*)X, (int64_t)d * es, (const char*)weight, (char*)Y, (int64_t)d * es, n, nvec, 1.f / d, eps, n_dev);
+    DASH_CUDA_TRY(cudaGetLastError());
+    return DASH_OK;
+}
+
+// U = Attn(LN(H)) (Eq. 1) into W.U: RMSNorm -> Q | K | V projection -> rotary embedding -> causal attention over the packed
+// active set -> output projection
+static int attention_branch(const dash_layer_cfg* cfg, const void* H_in, const int32_t* pos_in, const int32_t* cu_in, int S, int64_t n,
+                            int64_t max_seqlen, const StepWs& W, cudaStream_t st) {
+    const int es = cfg->dt == DASH_BF16 ? 2 : 4;
+    const bool bf = cfg->dt == DASH_BF16;
+    const int d = cfg->d, Hq = cfg->Hq, Hkv = cfg->Hkv, D = cfg->D;
+    const int64_t nq = (int64_t)(Hq + 2 * Hkv) * D;
+    const int32_t* n_dev = cu_in + S;            // true number of entering tokens lives on the device
+    int rc;
+    // LN (read as RMSNorm)
+    if ((rc = launch_rmsnorm(cfg->dt, H_in, cfg->rms_weight, W.Hn, n, d, cfg->rms_eps, n_dev, st)) != DASH_OK) return rc;
+    // Q | K | V = Hn Wqkv
+    if ((rc = gemm_rowmajor(cfg->dt, W.Hn, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, W.lt_ws, st)) != DASH_OK) return rc;
+    // rotary embedding on the Q and K heads
+    RopeFreq fr;
+    for (int i = 0; i < D / 2; ++i) fr.inv_freq[i] = pow(cfg->rope_base, -2.0 * i / D);
+    const int heads = Hq + Hkv;
+    if (bf && D == 128) rope_kernel<true, 128><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
+    else if (bf) rope_kernel<true, 64><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
+    else if (D == 128) rope_kernel<false, 128><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
+    else rope_kernel<false, 64><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
+    DASH_CUDA_TRY(cudaGetLastError());
+    // attention over the packed active set
+    rc = dash_varlen_attention(W.QKV, W.QKV + (int64_t)Hq * D * es, W.QKV + (int64_t)(Hq + Hkv) * D * es, W.O, nullptr, nq, nq, nq,
+                               (int64_t)Hq * D, cu_in, S, n, max_seqlen, Hq, Hkv, D, 1.0f / sqrtf((float)D), 1, cfg->dt,
+                               W.attn_ws, W.attn_bytes, st);
+    if (rc != DASH_OK) return rc;
+    // U = O Wo  (pre-residual attention output, Eq. 1)
+    return gemm_rowmajor(cfg->dt, W.O, (int64_t)Hq * D, cfg->Wo, d, W.U, d, n, d, (int64_t)Hq * D, W.lt_ws, st);
+}
+
+// r (and, threshold rule, the keep mask) from U and H, H~ = H + U into W.Ht; keep-count rule: the radix select on r
+static int score_and_select(const dash_layer_cfg* cfg, const void* H_in, const int32_t* cu_in, int S, int64_t n, float* r_out,
+                            uint8_t* mask_out, const StepWs& W, cudaStream_t st) {
+    const int d = cfg->d;
+    dash_threshold ft = {cfg->tau, cfg->keep_first, cfg->keep_last, cu_in, S, mask_out};
+    int rc = dash_delta_norm(W.U, H_in, n, d, d, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, r_out, W.Ht, d, nullptr,
+                             cfg->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr, cu_in + S, st);
+    if (rc != DASH_OK) return rc;
+    if (cfg->sel_mode == DASH_SEL_KEEP_COUNT)
+        rc = dash_select(r_out, n, cu_in, S, DASH_SEL_KEEP_COUNT, 0.f, cfg->keep_counts, cfg->keep_first, cfg->keep_last, mask_out,
+                         nullptr, 0, st);
+    return rc;
+}
+
+static bool block_cfg_ok(const dash_block_cfg* c) {
+    if (!c || !cfg_ok(&c->attn)) return false;
+    const int epv = c->attn.dt == DASH_BF16 ? 8 : 4;
+    if (c->m <= 0 || (c->m % epv) || !c->Wgu || !c->Wd || !c->rms2_weight) return false;
+    return c->attn.scatter_which == 2;
+}
+
+}  // namespace dash
+
 extern "C" int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, const int32_t* tok_index_in,
                                const int32_t* pos_in, const int32_t* cu_in, int S, int64_t n, int64_t max_seqlen,
                                void* x_full, void* H_next, int32_t* tok_index_next, int32_t* pos_next,
@@ -220,73 +337,94 @@ extern "C" int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, cons
     if (!cu_in || !cu_next) return DASH_ERR_INVALID_ARG;
     if (n > 0 && (!H_in || !pos_in || !tok_index_in || !x_full || !H_next || !tok_index_next || !pos_next || !r_out || !mask_out))
         return DASH_ERR_INVALID_ARG;
-    dash_layer_ws_layout L;
-    int rc = dash_layer_workspace(cfg, n, S, &L);
+    StepWs W;
+    int rc = carve_ws(cfg, n, S, ws, &W);
     if (rc != DASH_OK) return rc;
-    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < L.total) return DASH_ERR_WORKSPACE;
+    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < W.L.total) return DASH_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    char* w = (char*)ws;
     const int es = cfg->dt == DASH_BF16 ? 2 : 4;
-    const bool bf = cfg->dt == DASH_BF16;
-    const int d = cfg->d, Hq = cfg->Hq, Hkv = cfg->Hkv, D = cfg->D;
-    const int64_t nq = (int64_t)(Hq + 2 * Hkv) * D;
-    char *Hn = w + L.Hn, *QKV = w + L.QKV, *O = w + L.O, *U = w + L.U, *Ht = w + L.Ht;
-    char* lt_ws = w + L.scratch;
-    char* compact_ws = lt_ws + kLtWorkspace;
-    const size_t compact_bytes = align_up(dash_workspace_bytes(DASH_WS_COMPACT, n, S, 0, 0, 0, cfg->dt), 256);
-    char* attn_ws = compact_ws + compact_bytes;
-    const size_t attn_bytes = dash_workspace_bytes(DASH_WS_ATTENTION, n, S, Hq, Hkv, D, cfg->dt);
-    const int32_t* n_dev = cu_in + S;            // true number of entering tokens lives on the device
-
+    const int d = cfg->d;
     if (n > 0) {
         if (!aligned16(H_in) || !aligned16(x_full) || !aligned16(H_next) || !aligned16(cfg->Wqkv) || !aligned16(cfg->Wo) ||
             !aligned16(cfg->rms_weight))
             return DASH_ERR_INVALID_ARG;
-        // LN (read as RMSNorm)
-        const int nvec = d * es / 16;
-        if (bf) rmsnorm_kernel<true><<<rows_grid8(n), 256, 0, st>>>((const char*)H_in, (int64_t)d * es, (const char*)cfg->rms_weight, Hn, (int64_t)d * es, n, nvec, 1.f / d, cfg->rms_eps, n_dev);
-        else rmsnorm_kernel<false><<<rows_grid8(n), 256, 0, st>>>((const char*)H_in, (int64_t)d * es, (const char*)cfg->rms_weight, Hn, (int64_t)d * es, n, nvec, 1.f / d, cfg->rms_eps, n_dev);
-        DASH_CUDA_TRY(cudaGetLastError());
-        // Q | K | V = Hn Wqkv
-        if ((rc = gemm_rowmajor(cfg->dt, Hn, d, cfg->Wqkv, nq, QKV, nq, n, nq, d, lt_ws, st)) != DASH_OK) return rc;
-        // rotary embedding on the Q and K heads
-        RopeFreq fr;
-        for (int i = 0; i < D / 2; ++i) fr.inv_freq[i] = pow(cfg->rope_base, -2.0 * i / D);
-        const int heads = Hq + Hkv;
-        if (bf && D == 128) rope_kernel<true, 128><<<rows_grid8(n), 256, 0, st>>>(QKV, nq * es, pos_in, n, heads, fr, n_dev);
-        else if (bf) rope_kernel<true, 64><<<rows_grid8(n), 256, 0, st>>>(QKV, nq * es, pos_in, n, heads, fr, n_dev);
-        else if (D == 128) rope_kernel<false, 128><<<rows_grid8(n), 256, 0, st>>>(QKV, nq * es, pos_in, n, heads, fr, n_dev);
-        else rope_kernel<false, 64><<<rows_grid8(n), 256, 0, st>>>(QKV, nq * es, pos_in, n, heads, fr, n_dev);
-        DASH_CUDA_TRY(cudaGetLastError());
-        // attention over the packed active set
-        rc = dash_varlen_attention(QKV, QKV + (int64_t)Hq * D * es, QKV + (int64_t)(Hq + Hkv) * D * es, O, nullptr, nq, nq, nq,
-                                   (int64_t)Hq * D, cu_in, S, n, max_seqlen, Hq, Hkv, D, 1.0f / sqrtf((float)D), 1, cfg->dt,
-                                   attn_ws, attn_bytes, st);
-        if (rc != DASH_OK) return rc;
-        // U = O Wo  (pre-residual attention output, Eq. 1)
-        if ((rc = gemm_rowmajor(cfg->dt, O, (int64_t)Hq * D, cfg->Wo, d, U, d, n, d, (int64_t)Hq * D, lt_ws, st)) != DASH_OK) return rc;
+        if ((rc = attention_branch(cfg, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
         if (cfg->sel_mode == DASH_SEL_THRESHOLD && cfg->scatter_which == 2) {
             // r, H~ = H + U, the halting rule, the scatter of H~ and the compaction of the rows that stay, in one pass
-            return launch_delta_tail(U, H_in, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau, cfg->keep_first, cfg->keep_last,
-                                     cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out, tok_index_next, pos_next,
-                                     cu_next, n_next_dev, compact_ws, compact_bytes, st);
+            return launch_delta_tail(W.U, H_in, nullptr, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau, cfg->keep_first,
+                                     cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out, tok_index_next,
+                                     pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, st);
         }
-        // r, H~ = H + U, and (threshold mode) the halting rule in the same pass
-        dash_threshold ft = {cfg->tau, cfg->keep_first, cfg->keep_last, cu_in, S, mask_out};
-        rc = dash_delta_norm(U, H_in, n, d, d, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, r_out, Ht, d, nullptr,
-                             cfg->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr, n_dev, st);
-        if (rc != DASH_OK) return rc;
-        if (cfg->sel_mode == DASH_SEL_KEEP_COUNT) {
-            rc = dash_select(r_out, n, cu_in, S, DASH_SEL_KEEP_COUNT, 0.f, cfg->keep_counts, cfg->keep_first, cfg->keep_last,
-                             mask_out, nullptr, 0, st);
-            if (rc != DASH_OK) return rc;
-        }
+        if ((rc = score_and_select(cfg, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;
         // updated states reach the full-length output (halted tokens stay frozen there from now on)
-        rc = dash_scatter(Ht, n, (int64_t)d * es, (int64_t)d * es, tok_index_in, mask_out, cfg->scatter_which, n_dev, x_full,
+        rc = dash_scatter(W.Ht, n, (int64_t)d * es, (int64_t)d * es, tok_index_in, mask_out, cfg->scatter_which, cu_in + S, x_full,
                           (int64_t)d * es, st);
         if (rc != DASH_OK) return rc;
     }
-    dash_rows rows = {Ht, H_next, (int64_t)d * es, (int64_t)d * es, (int64_t)d * es};
+    dash_rows rows = {W.Ht, H_next, (int64_t)d * es, (int64_t)d * es, (int64_t)d * es};
     return dash_compact(mask_out, n, cu_in, S, &rows, n > 0 ? 1 : 0, pos_in, pos_next, tok_index_in, tok_index_next, nullptr,
-                        cu_next, n_next_dev, compact_ws, compact_bytes, st);
+                        cu_next, n_next_dev, W.compact_ws, W.compact_bytes, st);
+}
+
+extern "C" int dash_block_workspace(const dash_block_cfg* cfg, int64_t n, int S, dash_block_ws_layout* out) {
+    if (!block_cfg_ok(cfg) || n < 0 || S < 1 || !out) return DASH_ERR_INVALID_ARG;
+    int rc = dash_layer_workspace(&cfg->attn, n, S, &out->attn);
+    if (rc != DASH_OK) return rc;
+    const size_t es = cfg->attn.dt == DASH_BF16 ? 2 : 4;
+    size_t off = align_up(out->attn.total, 256);
+    out->GU = off;  off += align_up((size_t)n * 2 * cfg->m * es, 256);
+    out->ACT = off; off += align_up((size_t)n * cfg->m * es, 256);
+    out->F = off;   off += align_up((size_t)n * cfg->attn.d * es, 256);
+    out->total = off;
+    return DASH_OK;
+}
+
+extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, const int32_t* tok_index_in,
+                               const int32_t* pos_in, const int32_t* cu_in, int S, int64_t n, int64_t max_seqlen,
+                               void* x_full, void* H_next, int32_t* tok_index_next, int32_t* pos_next,
+                               int32_t* cu_next, int32_t* n_next_dev, float* r_out, uint8_t* mask_out,
+                               void* ws, size_t ws_bytes, void* stream) {
+    if (!block_cfg_ok(cfg) || n < 0 || S < 1 || max_seqlen < 0 || max_seqlen > n) return DASH_ERR_INVALID_ARG;
+    if (!cu_in || !cu_next) return DASH_ERR_INVALID_ARG;
+    if (n > 0 && (!H_in || !pos_in || !tok_index_in || !x_full || !H_next || !tok_index_next || !pos_next || !r_out || !mask_out))
+        return DASH_ERR_INVALID_ARG;
+    const dash_layer_cfg* a = &cfg->attn;
+    dash_block_ws_layout BL;
+    int rc = dash_block_workspace(cfg, n, S, &BL);
+    if (rc != DASH_OK) return rc;
+    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < BL.total) return DASH_ERR_WORKSPACE;
+    StepWs W;
+    if ((rc = carve_ws(a, n, S, ws, &W)) != DASH_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int es = a->dt == DASH_BF16 ? 2 : 4;
+    const int d = a->d, m = cfg->m;
+    char *GU = (char*)ws + BL.GU, *ACT = (char*)ws + BL.ACT, *F = (char*)ws + BL.F;
+    if (n == 0) {
+        return dash_compact(mask_out, 0, cu_in, S, nullptr, 0, pos_in, pos_next, tok_index_in, tok_index_next, nullptr, cu_next, n_next_dev,
+                            W.compact_ws, W.compact_bytes, st);
+    }
+    if (!aligned16(H_in) || !aligned16(x_full) || !aligned16(H_next) || !aligned16(a->Wqkv) || !aligned16(a->Wo) || !aligned16(a->rms_weight) ||
+        !aligned16(cfg->Wgu) || !aligned16(cfg->Wd) || !aligned16(cfg->rms2_weight))
+        return DASH_ERR_INVALID_ARG;
+    const int32_t* n_dev = cu_in + S;
+    // U = Attn(LN(H)); score and selection from U; H~ = H + U
+    if ((rc = attention_branch(a, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
+    if ((rc = score_and_select(a, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;
+    // F = FFN(LN(H~)): gate | up projection, silu(gate) * up, down projection
+    if ((rc = launch_rmsnorm(a->dt, W.Ht, cfg->rms2_weight, W.Hn, n, d, a->rms_eps, n_dev, st)) != DASH_OK) return rc;
+    if ((rc = gemm_rowmajor(a->dt, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, GU, 2 * (int64_t)m, n, 2 * (int64_t)m, d, W.lt_ws, st)) != DASH_OK) return rc;
+    {
+        const int64_t total = n * (int64_t)(m / (16 / es));
+        int64_t blocks = (total + 255) / 256, cap = (int64_t)sm_count() * 16;
+        if (blocks > cap) blocks = cap;
+        if (a->dt == DASH_BF16) swiglu_kernel<true><<<(int)blocks, 256, 0, st>>>(GU, 2 * (int64_t)m * es, ACT, (int64_t)m * es, n, m, n_dev);
+        else swiglu_kernel<false><<<(int)blocks, 256, 0, st>>>(GU, 2 * (int64_t)m * es, ACT, (int64_t)m * es, n, m, n_dev);
+        DASH_CUDA_TRY(cudaGetLastError());
+    }
+    if ((rc = gemm_rowmajor(a->dt, ACT, m, cfg->Wd, d, F, d, n, d, m, W.lt_ws, st)) != DASH_OK) return rc;
+    // H' = H~ + F to x_full (every entering token: H' is also the last updated value of the tokens that halt here) and,
+    // for the tokens that stay, to the next block's packed buffer -- one pass, keep decisions taken from mask_out
+    return launch_delta_tail(F, W.Ht, mask_out, n, d, a->dt, a->norm_mode, a->norm_eps, a->tau, a->keep_first, a->keep_last, cu_in, S,
+                             tok_index_in, pos_in, x_full, H_next, nullptr, nullptr, tok_index_next, pos_next, cu_next, n_next_dev,
+                             W.compact_ws, W.compact_bytes, st);
 }

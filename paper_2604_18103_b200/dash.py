@@ -28,6 +28,7 @@ EXPORTS = [
     "dash_status_string", "dash_check_status", "dash_keep_count", "dash_flops_per_layer", "dash_flops_speedup",
     "dash_delta_norm", "dash_select", "dash_compact", "dash_scatter", "dash_varlen_attention",
     "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes", "dash_compact_static",
+    "dash_block_workspace", "dash_block_step",
 ]
 COMPACT_STATIC_MAX_ROWS = 1 << 20
 
@@ -53,6 +54,14 @@ class LayerCfg(Structure):
 class LayerWsLayout(Structure):
     _fields_ = [("Hn", c_size_t), ("QKV", c_size_t), ("O", c_size_t), ("U", c_size_t), ("Ht", c_size_t),
                 ("scratch", c_size_t), ("total", c_size_t)]
+
+
+class BlockCfg(Structure):
+    _fields_ = [("attn", LayerCfg), ("m", c_int), ("Wgu", c_void_p), ("Wd", c_void_p), ("rms2_weight", c_void_p)]
+
+
+class BlockWsLayout(Structure):
+    _fields_ = [("attn", LayerWsLayout), ("GU", c_size_t), ("ACT", c_size_t), ("F", c_size_t), ("total", c_size_t)]
 
 
 _lib = None
@@ -90,6 +99,10 @@ def lib() -> ctypes.CDLL:
                                                                           c_void_p, c_size_t, c_void_p]
         L.dash_layer_workspace.argtypes = [POINTER(LayerCfg), c_int64, c_int, POINTER(LayerWsLayout)]
         L.dash_layer_step.argtypes = [POINTER(LayerCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
+                                      c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                      c_void_p, c_size_t, c_void_p]
+        L.dash_block_workspace.argtypes = [POINTER(BlockCfg), c_int64, c_int, POINTER(BlockWsLayout)]
+        L.dash_block_step.argtypes = [POINTER(BlockCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_size_t, c_void_p]
         L.dash_workspace_bytes.restype = c_size_t
@@ -297,3 +310,39 @@ def dash_layer_step(layer: Layer, H_in, tok_index_in, pos_in, cu_in, max_seqlen:
                                int(max_seqlen), _p(x_full), _p(H_next), _p(tok_index_next), _p(pos_next), _p(cu_next), _p(n_next),
                                _p(r_out), _p(mask_out), _p(ws), ws.numel(), _stream())
     _check(st, "dash_layer_step")
+
+
+# ---- the whole block, feed-forward included -------------------------------------------
+class Block:
+    """Device-resident weights and configuration of one whole block (attention + gated FFN) for dash_block_step."""
+
+    def __init__(self, shape, weights, device, **layer_kwargs):
+        self.layer = Layer(shape, weights, device, **layer_kwargs)
+        self.shape = shape
+        self.Wgu = torch.cat([weights["Wg"], weights["Wu"]], dim=1).contiguous().to(device)
+        self.Wd = weights["Wd"].contiguous().to(device)
+        self.rms2_w = weights["rms2_w"].contiguous().to(device)
+        self.cfg = BlockCfg(self.layer.cfg, shape.m, self.Wgu.data_ptr(), self.Wd.data_ptr(), self.rms2_w.data_ptr())
+
+    def set_tau(self, tau: float):
+        self.cfg.attn.tau = float(tau)
+
+    def set_keep_counts(self, keep_counts: Optional[torch.Tensor], sel_mode: int):
+        self.keep_counts = keep_counts
+        self.cfg.attn.sel_mode = sel_mode
+        self.cfg.attn.keep_counts = keep_counts.data_ptr() if keep_counts is not None else None
+
+
+def dash_block_workspace(block: Block, n: int, S: int) -> BlockWsLayout:
+    out = BlockWsLayout()
+    _check(lib().dash_block_workspace(ctypes.byref(block.cfg), n, S, ctypes.byref(out)), "dash_block_workspace")
+    return out
+
+
+def dash_block_step(block: Block, H_in, tok_index_in, pos_in, cu_in, max_seqlen: int, x_full, H_next, tok_index_next, pos_next,
+                    cu_next, n_next, r_out, mask_out, ws):
+    n = H_in.shape[0]
+    st = lib().dash_block_step(ctypes.byref(block.cfg), _p(H_in), _p(tok_index_in), _p(pos_in), _p(cu_in), cu_in.numel() - 1, n,
+                               int(max_seqlen), _p(x_full), _p(H_next), _p(tok_index_next), _p(pos_next), _p(cu_next), _p(n_next),
+                               _p(r_out), _p(mask_out), _p(ws), ws.numel(), _stream())
+    _check(st, "dash_block_step")
