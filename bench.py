@@ -44,8 +44,8 @@ from paper_2604_18103_b200 import workloads as wl  # noqa: E402
 METRIC = "active_token_prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 L2_FLUSH_BYTES = 256 << 20
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch (ncu, profiles/attention_kernel_cfg2_8192.md); null where
-# no capture of the current kernel exists
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch (from the committed ncu summary of this kernel and
+# workload); null where no capture of the current kernel exists
 ATTN_TRAFFIC = {"cfg2": 94.74e6}
 
 
