@@ -51,7 +51,13 @@ typedef enum { DASH_F32 = 0, DASH_BF16 = 1 } dash_dtype;
 /* REL: ||U_t|| / ||H_t|| (the "relative" delta-attention of Fig. 1);
  * ABS: ||U_t||           (Eq. 2). */
 typedef enum { DASH_NORM_REL = 0, DASH_NORM_ABS = 1 } dash_norm_mode;
-typedef enum { DASH_SEL_THRESHOLD = 0, DASH_SEL_KEEP_COUNT = 1 } dash_sel_mode;
+/* The _HALT_HIGH variants are the paper's direction ablation ("High Delta_attn"): the same rules on the
+ * negated scores -- a token halts iff r > tau, or the smallest scores stay. */
+typedef enum { DASH_SEL_THRESHOLD = 0, DASH_SEL_KEEP_COUNT = 1,
+               DASH_SEL_THRESHOLD_HALT_HIGH = 2, DASH_SEL_KEEP_COUNT_HALT_HIGH = 3 } dash_sel_mode;
+/* Score of dash_block_step: the attention branch's update (Eq. 2, the method) or the change over the whole
+ * block, ||H' - H|| (the paper's ablation of the delta signal). */
+typedef enum { DASH_SIGNAL_ATTN = 0, DASH_SIGNAL_BLOCK = 1 } dash_signal;
 
 #define DASH_MAX_ROW_STREAMS 8
 
@@ -101,6 +107,8 @@ int dash_delta_norm(const void* U, const void* H, int64_t n, int d, int64_t ldU,
  * KEEP_COUNT: per sequence s, keep_counts[s] (device int32 [S]) tokens stay in
  *   total: the protected ones plus the largest scores of the others; ties at
  *   the cut are broken toward the lower index; NaN ranks as +inf.
+ * THRESHOLD_HALT_HIGH / KEEP_COUNT_HALT_HIGH: the same on -r (random halting needs no mode:
+ *   pass random scores).
  * r: device fp32 [n]; cu_seqlens: device int32 [S+1] over the current packed
  * order; mask_out: device u8 [n] (1 = stays active). */
 int dash_select(const float* r, int64_t n, const int32_t* cu_seqlens, int S,
@@ -234,6 +242,7 @@ typedef struct {
     const void*  Wgu;              /* [d, 2 m]: columns = Wg | Wu */
     const void*  Wd;               /* [m, d] */
     const void*  rms2_weight;      /* [d]: weight of the norm in front of the FFN (attn.rms_eps is used) */
+    dash_signal  signal;           /* what the score measures */
 } dash_block_cfg;
 typedef struct {
     dash_layer_ws_layout attn;

@@ -133,7 +133,7 @@ THRESHOLD, KEEP_COUNT = 0, 1
 
 
 def select(r, cu, mode: int, tau: float = 0.0, keep_counts: Optional[Sequence[int]] = None,
-           keep_first: int = 0, keep_last: int = 0) -> np.ndarray:
+           keep_first: int = 0, keep_last: int = 0, halt_high: bool = False) -> np.ndarray:
     """Keep mask (1 = stays active) from the scores r, per sequence.
 
     Protected tokens (first keep_first / last keep_last of each sequence in its
@@ -143,6 +143,8 @@ def select(r, cu, mode: int, tau: float = 0.0, keep_counts: Optional[Sequence[in
     KEEP_COUNT: Eq. 3, S* = TopK(S, K, Delta): K_s tokens of sequence s stay in
       total -- the protected ones plus the K_s - n_protected largest scores of
       the others, ties broken toward the lower index, NaN ranked as +inf.
+    halt_high (the paper's direction ablation, "High Delta_attn"): the rule runs on the negated
+    scores -- a token halts iff r_t > tau, or the K_s smallest scores stay.
     """
     r = np.asarray(r, dtype=np.float32)
     cu = i32(cu)
@@ -156,8 +158,10 @@ def select(r, cu, mode: int, tau: float = 0.0, keep_counts: Optional[Sequence[in
         if keep_last > 0:
             protected[max(0, ns - keep_last):] = True
         rs = r[a:b]
+        if halt_high:
+            rs = -rs
         if mode == THRESHOLD:
-            halted = (rs < np.float32(tau)) & ~protected
+            halted = (rs < np.float32(-tau if halt_high else tau)) & ~protected
             mask[a:b] = (~halted).astype(np.uint8)
         else:
             K = int(keep_counts[s])
@@ -329,18 +333,25 @@ def ffn_swiglu(X, Wg, Wu, Wd) -> np.ndarray:
 def block_step(H, weights: Dict[str, object], cu, pos, shape, norm_mode: int = REL,
                sel_mode: int = THRESHOLD, tau: float = 0.0, keep_counts=None,
                keep_first: int = 0, keep_last: int = 0, eps: float = 1e-12,
-               attn_rows=None) -> Dict[str, object]:
+               attn_rows=None, signal: str = "attn", halt_high: bool = False) -> Dict[str, object]:
     """One whole block of Alg. 1 on the packed active tokens: U = Attn(LN(H)); H~ = H + U;
     H' = H~ + FFN(LN(H~)); the score is taken from U, the selection from the score; the tokens that
     stay carry H' into the next block, and H' is also the last updated value of the tokens that halt
     here (Sec. 3.4).  `weights` holds the attention weights of layer_step plus Wg, Wu, Wd, rms2_w.
-    With attn_rows given only those rows are evaluated (no selection)."""
+    With attn_rows given only those rows are evaluated (no selection).
+    signal = "block" (the paper's ablation of the delta signal): the score is the change over the whole
+    block, ||H' - H|| (relative: / ||H||), instead of the attention branch's ||U||."""
     out = layer_step(H, weights, cu, pos, shape, norm_mode, sel_mode, tau, keep_counts, keep_first, keep_last, eps, attn_rows)
     Hn2 = rmsnorm(out["Ht"], weights["rms2_w"], shape.rms_eps)
     out["F"] = ffn_swiglu(Hn2, weights["Wg"], weights["Wu"], weights["Wd"])
     out["H1"] = out["Ht"] + out["F"]
+    Hsel = f64(H) if attn_rows is None else f64(H)[np.asarray(attn_rows, dtype=np.int64)]
+    if signal == "block":
+        out["r"] = delta_norm(out["H1"] - Hsel, Hsel, norm_mode, eps)
     if attn_rows is not None:
         return out
+    if signal == "block" or halt_high:
+        out["mask"] = select(out["r"], cu, sel_mode, tau, keep_counts, keep_first, keep_last, halt_high)
     out.update(compact(out["mask"], cu, rows=[out["H1"]], pos_in=pos))
     return out
 

@@ -105,14 +105,15 @@ delta_norm_kernel(const char* __restrict__ U, const char* __restrict__ H, int64_
 // step 2: halting rule
 // ---------------------------------------------------------------------------
 __global__ void select_threshold_kernel(const float* __restrict__ r, int64_t n, const int32_t* __restrict__ cu, int S,
-                                        float tau, int keep_first, int keep_last, uint8_t* __restrict__ mask) {
+                                        float tau, int keep_first, int keep_last, uint8_t* __restrict__ mask, int halt_high) {
     int64_t total = cu[S];
     if (total < n) n = total;
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < n; t += (int64_t)gridDim.x * blockDim.x) {
         int s = find_seq(cu, S, (int)t);
         int local = (int)t - cu[s], len = cu[s + 1] - cu[s];
         bool prot = (local < keep_first) || (local >= len - keep_last);
-        mask[t] = (prot || !(r[t] < tau)) ? 1 : 0;
+        const bool halted = halt_high ? (r[t] > tau) : (r[t] < tau);      // NaN compares false: stays
+        mask[t] = (prot || !halted) ? 1 : 0;
     }
 }
 
@@ -159,7 +160,7 @@ __device__ __forceinline__ int block_excl_scan_1024(int v, int* s_warp, int* tot
 __global__ void __launch_bounds__(1024)
 select_keep_count_kernel(const float* __restrict__ r, const int32_t* __restrict__ cu, int S,
                          const int32_t* __restrict__ keep_counts, int keep_first, int keep_last,
-                         uint8_t* __restrict__ mask) {
+                         uint8_t* __restrict__ mask, int halt_high) {
     __shared__ int hist[256];
     __shared__ int s_warp[33];
     __shared__ uint32_t s_prefix;
@@ -186,7 +187,7 @@ select_keep_count_kernel(const float* __restrict__ r, const int32_t* __restrict_
         for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
         __syncthreads();
         for (int t = e0 + threadIdx.x; t < e1; t += blockDim.x) {
-            uint32_t key = order_key(r[t]);
+            uint32_t key = order_key(halt_high ? -r[t] : r[t]);
             if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
         }
         __syncthreads();
@@ -210,11 +211,11 @@ select_keep_count_kernel(const float* __restrict__ r, const int32_t* __restrict_
     const int per = (n_el + blockDim.x - 1) / blockDim.x;
     const int t0 = min(e0 + (int)threadIdx.x * per, e1), t1 = min(t0 + per, e1);
     int ties = 0;
-    for (int t = t0; t < t1; ++t) ties += (order_key(r[t]) == cut);
+    for (int t = t0; t < t1; ++t) ties += (order_key(halt_high ? -r[t] : r[t]) == cut);
     int total;
     int rank = block_excl_scan_1024(ties, s_warp, &total);
     for (int t = t0; t < t1; ++t) {
-        uint32_t key = order_key(r[t]);
+        uint32_t key = order_key(halt_high ? -r[t] : r[t]);
         uint8_t v = 0;
         if (key > cut) v = 1;
         else if (key == cut) { v = rank < remaining; ++rank; }
@@ -638,19 +639,20 @@ extern "C" int dash_select(const float* r, int64_t n, const int32_t* cu_seqlens,
                            void* ws, size_t ws_bytes, void* stream) {
     (void)ws; (void)ws_bytes;
     if (n < 0 || S < 1 || !cu_seqlens || keep_first < 0 || keep_last < 0) return DASH_ERR_INVALID_ARG;
-    if (mode != DASH_SEL_THRESHOLD && mode != DASH_SEL_KEEP_COUNT) return DASH_ERR_INVALID_ARG;
+    if (mode < DASH_SEL_THRESHOLD || mode > DASH_SEL_KEEP_COUNT_HALT_HIGH) return DASH_ERR_INVALID_ARG;
+    const int halt_high = (mode == DASH_SEL_THRESHOLD_HALT_HIGH || mode == DASH_SEL_KEEP_COUNT_HALT_HIGH) ? 1 : 0;
     if (n > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
     if (n == 0) return DASH_OK;
     if (!r || !mask_out) return DASH_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    if (mode == DASH_SEL_THRESHOLD) {
+    if (mode == DASH_SEL_THRESHOLD || mode == DASH_SEL_THRESHOLD_HALT_HIGH) {
         int grid = (int)((n + 255) / 256);
         int cap = sm_count() * 8;
         if (grid > cap) grid = cap;
-        select_threshold_kernel<<<grid, 256, 0, st>>>(r, n, cu_seqlens, S, tau, keep_first, keep_last, mask_out);
+        select_threshold_kernel<<<grid, 256, 0, st>>>(r, n, cu_seqlens, S, tau, keep_first, keep_last, mask_out, halt_high);
     } else {
         if (!keep_counts) return DASH_ERR_INVALID_ARG;
-        select_keep_count_kernel<<<S, 1024, 0, st>>>(r, cu_seqlens, S, keep_counts, keep_first, keep_last, mask_out);
+        select_keep_count_kernel<<<S, 1024, 0, st>>>(r, cu_seqlens, S, keep_counts, keep_first, keep_last, mask_out, halt_high);
     }
     DASH_CUDA_TRY(cudaGetLastError());
     return DASH_OK;

@@ -213,8 +213,8 @@ static bool cfg_ok(const dash_layer_cfg* c) {
     if ((c->d % 8) || (c->Hq % c->Hkv)) return false;
     if (c->dt != DASH_F32 && c->dt != DASH_BF16) return false;
     if (!c->Wqkv || !c->Wo || !c->rms_weight) return false;
-    if (c->sel_mode != DASH_SEL_THRESHOLD && c->sel_mode != DASH_SEL_KEEP_COUNT) return false;
-    if (c->sel_mode == DASH_SEL_KEEP_COUNT && !c->keep_counts) return false;
+    if (c->sel_mode < DASH_SEL_THRESHOLD || c->sel_mode > DASH_SEL_KEEP_COUNT_HALT_HIGH) return false;
+    if ((c->sel_mode == DASH_SEL_KEEP_COUNT || c->sel_mode == DASH_SEL_KEEP_COUNT_HALT_HIGH) && !c->keep_counts) return false;
     if (c->keep_first < 0 || c->keep_last < 0) return false;
     if (c->scatter_which != 0 && c->scatter_which != 2) return false;
     if (!(c->rope_base > 0.0)) return false;
@@ -313,8 +313,8 @@ static int score_and_select(const dash_layer_cfg* cfg, const void* H_in, const i
     int rc = dash_delta_norm(W.U, H_in, n, d, d, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, r_out, W.Ht, d, nullptr,
                              cfg->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr, cu_in + S, st);
     if (rc != DASH_OK) return rc;
-    if (cfg->sel_mode == DASH_SEL_KEEP_COUNT)
-        rc = dash_select(r_out, n, cu_in, S, DASH_SEL_KEEP_COUNT, 0.f, cfg->keep_counts, cfg->keep_first, cfg->keep_last, mask_out,
+    if (cfg->sel_mode != DASH_SEL_THRESHOLD)
+        rc = dash_select(r_out, n, cu_in, S, cfg->sel_mode, cfg->tau, cfg->keep_counts, cfg->keep_first, cfg->keep_last, mask_out,
                          nullptr, 0, st);
     return rc;
 }
@@ -323,6 +323,8 @@ static bool block_cfg_ok(const dash_block_cfg* c) {
     if (!c || !cfg_ok(&c->attn)) return false;
     const int epv = c->attn.dt == DASH_BF16 ? 8 : 4;
     if (c->m <= 0 || (c->m % epv) || !c->Wgu || !c->Wd || !c->rms2_weight) return false;
+    if (c->signal != DASH_SIGNAL_ATTN && c->signal != DASH_SIGNAL_BLOCK) return false;
+    if (c->signal == DASH_SIGNAL_BLOCK && 2 * c->m < c->attn.d) return false;      // U + F is formed in the gate | up buffer
     return c->attn.scatter_which == 2;
 }
 
@@ -409,7 +411,7 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
     const int32_t* n_dev = cu_in + S;
     // U = Attn(LN(H)); score and selection from U; H~ = H + U
     if ((rc = attention_branch(a, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
-    if ((rc = score_and_select(a, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;
+    if ((rc = score_and_select(a, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;   // also leaves H~ in W.Ht
     // F = FFN(LN(H~)): gate | up projection, silu(gate) * up, down projection
     if ((rc = launch_rmsnorm(a->dt, W.Ht, cfg->rms2_weight, W.Hn, n, d, a->rms_eps, n_dev, st)) != DASH_OK) return rc;
     if ((rc = gemm_rowmajor(a->dt, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, GU, 2 * (int64_t)m, n, 2 * (int64_t)m, d, W.lt_ws, st)) != DASH_OK) return rc;
@@ -422,6 +424,17 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         DASH_CUDA_TRY(cudaGetLastError());
     }
     if ((rc = gemm_rowmajor(a->dt, ACT, m, cfg->Wd, d, F, d, n, d, m, W.lt_ws, st)) != DASH_OK) return rc;
+    if (cfg->signal == DASH_SIGNAL_BLOCK) {
+        // ablation: score = change over the whole block, H' - H = U + F (formed in the gate | up buffer, free by now)
+        if ((rc = dash_delta_norm(F, W.U, n, d, d, d, a->dt, DASH_NORM_ABS, a->norm_eps, r_out, GU, d, nullptr, nullptr, n_dev, st)) != DASH_OK) return rc;
+        dash_threshold ft = {a->tau, a->keep_first, a->keep_last, cu_in, S, mask_out};
+        rc = dash_delta_norm(GU, H_in, n, d, d, d, a->dt, a->norm_mode, a->norm_eps, r_out, nullptr, d, nullptr,
+                             a->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr, n_dev, st);
+        if (rc != DASH_OK) return rc;
+        if (a->sel_mode != DASH_SEL_THRESHOLD &&
+            (rc = dash_select(r_out, n, cu_in, S, a->sel_mode, a->tau, a->keep_counts, a->keep_first, a->keep_last, mask_out, nullptr, 0, st)) != DASH_OK)
+            return rc;
+    }
     // H' = H~ + F to x_full (every entering token: H' is also the last updated value of the tokens that halt here) and,
     // for the tokens that stay, to the next block's packed buffer -- one pass, keep decisions taken from mask_out
     return launch_delta_tail(F, W.Ht, mask_out, n, d, a->dt, a->norm_mode, a->norm_eps, a->tau, a->keep_first, a->keep_last, cu_in, S,

@@ -17,7 +17,8 @@ import torch
 
 F32, BF16 = 0, 1
 NORM_REL, NORM_ABS = 0, 1
-SEL_THRESHOLD, SEL_KEEP_COUNT = 0, 1
+SEL_THRESHOLD, SEL_KEEP_COUNT, SEL_THRESHOLD_HALT_HIGH, SEL_KEEP_COUNT_HALT_HIGH = 0, 1, 2, 3
+SIGNAL_ATTN, SIGNAL_BLOCK = 0, 1
 WS_SELECT, WS_COMPACT, WS_ATTENTION = 0, 1, 2
 OK = 0
 
@@ -57,7 +58,7 @@ class LayerWsLayout(Structure):
 
 
 class BlockCfg(Structure):
-    _fields_ = [("attn", LayerCfg), ("m", c_int), ("Wgu", c_void_p), ("Wd", c_void_p), ("rms2_weight", c_void_p)]
+    _fields_ = [("attn", LayerCfg), ("m", c_int), ("Wgu", c_void_p), ("Wd", c_void_p), ("rms2_weight", c_void_p), ("signal", c_int)]
 
 
 class BlockWsLayout(Structure):
@@ -316,13 +317,13 @@ def dash_layer_step(layer: Layer, H_in, tok_index_in, pos_in, cu_in, max_seqlen:
 class Block:
     """Device-resident weights and configuration of one whole block (attention + gated FFN) for dash_block_step."""
 
-    def __init__(self, shape, weights, device, **layer_kwargs):
+    def __init__(self, shape, weights, device, signal=SIGNAL_ATTN, **layer_kwargs):
         self.layer = Layer(shape, weights, device, **layer_kwargs)
         self.shape = shape
         self.Wgu = torch.cat([weights["Wg"], weights["Wu"]], dim=1).contiguous().to(device)
         self.Wd = weights["Wd"].contiguous().to(device)
         self.rms2_w = weights["rms2_w"].contiguous().to(device)
-        self.cfg = BlockCfg(self.layer.cfg, shape.m, self.Wgu.data_ptr(), self.Wd.data_ptr(), self.rms2_w.data_ptr())
+        self.cfg = BlockCfg(self.layer.cfg, shape.m, self.Wgu.data_ptr(), self.Wd.data_ptr(), self.rms2_w.data_ptr(), signal)
 
     def set_tau(self, tau: float):
         self.cfg.attn.tau = float(tau)

@@ -139,3 +139,35 @@ def test_block_step_qwen_shape_sampled_rows():
     far = np.abs(ref["r"].astype(np.float64) - tau) > BAND
     assert np.array_equal(mask[rows][far], (~(ref["r"] < np.float32(tau))).astype(np.uint8)[far])
     assert torch.equal(b.H_next[:K].cpu(), x_full.cpu()[np.flatnonzero(mask)])
+
+
+def test_block_step_block_signal_and_high_direction_ablations():
+    """The paper's ablations as modes: score from the change over the whole block; halting the high scores."""
+    w = wl.config2(T=700, seed=35, shape=wl.MINI)
+    sh, T = w.shape, w.T
+    H, W = w.tensors["H"], _weights(sh, 35)
+    pos = wl.positions(w.cu)
+    tok = torch.arange(T, dtype=torch.int32, device=DEV)
+    # block signal, threshold rule
+    ref0 = oc.block_step(H, W, w.cu, pos, sh, tau=0.0, signal="block")
+    tau = oc.kth_largest(ref0["r"], T // 2)
+    ref = oc.block_step(H, W, w.cu, pos, sh, tau=tau, signal="block")
+    block = dash.Block(sh, W, DEV, signal=dash.SIGNAL_BLOCK, tau=tau)
+    b = BlockBuffers(block, T, 1)
+    x_full = torch.zeros(T, sh.d, dtype=sh.dtype, device=DEV)
+    run_block(block, H.to(DEV), tok, pos.to(DEV), w.cu.to(DEV), T, x_full, b)
+    r_gpu, mask = b.r.cpu().numpy(), b.mask.cpu().numpy()
+    assert np.max(np.abs(r_gpu - ref["r"]) / ref["r"]) < 2e-2
+    check_mask(mask, r_gpu, ref["r"], tau, w.cu)
+    assert_close_h1(x_full.float().cpu().numpy(), ref["H1"], "H' (x_full)")
+    k = int(b.n_next.item())
+    assert k == int(mask.sum()) and torch.equal(b.H_next[:k].cpu(), x_full.cpu()[np.flatnonzero(mask)])
+    # attention signal, the K smallest scores stay
+    K = T // 3
+    kc = torch.tensor([K], dtype=torch.int32, device=DEV)
+    block2 = dash.Block(sh, W, DEV, sel_mode=dash.SEL_KEEP_COUNT_HALT_HIGH, keep_counts=kc)
+    run_block(block2, H.to(DEV), tok, pos.to(DEV), w.cu.to(DEV), T, x_full, b)
+    r2, m2 = b.r.cpu().numpy(), b.mask.cpu().numpy()
+    assert int(b.n_next.item()) == K
+    assert np.array_equal(m2, oc.select(r2, w.cu, oc.KEEP_COUNT, keep_counts=[K], halt_high=True))
+    assert r2[m2 == 1].max() <= r2[m2 == 0].min()                           # the low scores stay, the high ones halt

@@ -118,6 +118,23 @@ def test_select_matches_oracle(lengths):
             assert np.array_equal(m.cpu().numpy(), ref), (lengths, kf, kl, frac)
 
 
+def test_select_high_direction_matches_oracle():
+    lengths = [300, 0, 1700, 1]
+    cu = wl.cu_from_lengths(lengths)
+    n = int(cu[-1])
+    g = torch.Generator().manual_seed(13)
+    r = torch.rand(n, generator=g)
+    r[5] = float("nan")
+    rd, cud = r.to(DEV), cu.to(DEV)
+    m = dash.dash_select(rd, cud, dash.SEL_THRESHOLD_HALT_HIGH, tau=0.6, keep_first=4, keep_last=2)
+    assert np.array_equal(m.cpu().numpy(), oc.select(r.numpy(), cu, oc.THRESHOLD, tau=0.6, keep_first=4, keep_last=2, halt_high=True))
+    K = [100, 0, 1234, 1]
+    m = dash.dash_select(rd, cud, dash.SEL_KEEP_COUNT_HALT_HIGH, keep_counts=torch.tensor(K, dtype=torch.int32, device=DEV), keep_first=4, keep_last=2)
+    ref = oc.select(r.numpy(), cu, oc.KEEP_COUNT, keep_counts=K, keep_first=4, keep_last=2, halt_high=True)
+    assert np.array_equal(m.cpu().numpy(), ref)
+    assert m.cpu().numpy()[5] == 1                                           # NaN stays in either direction
+
+
 def test_select_all_equal_scores_keeps_lowest_indices():
     n = 4096
     r = torch.full((n,), 0.25)

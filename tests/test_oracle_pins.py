@@ -125,6 +125,29 @@ def test_select_brute_force_tiny_and_ties():
     assert oc.select(rn, c3, oc.KEEP_COUNT, keep_counts=[1]).tolist() == [0, 1, 0]
 
 
+def test_select_high_direction_is_the_complement_rule():
+    g = torch.Generator().manual_seed(17)
+    r = torch.rand(300, generator=g).numpy().astype(np.float32)            # no ties
+    cu = np.array([0, 120, 120, 300], dtype=np.int32)
+    # threshold: away from equality the two directions are complements
+    tau = 0.37
+    lo = oc.select(r, cu, oc.THRESHOLD, tau=tau)
+    hi = oc.select(r, cu, oc.THRESHOLD, tau=tau, halt_high=True)
+    assert np.array_equal(hi, 1 - lo)
+    assert np.array_equal(hi, (r <= np.float32(tau)).astype(np.uint8))     # halts iff r > tau
+    # keep-count: keeping the K smallest == halting the n - K largest
+    K = [50, 0, 77]
+    hi_k = oc.select(r, cu, oc.KEEP_COUNT, keep_counts=K, halt_high=True)
+    lo_k = oc.select(r, cu, oc.KEEP_COUNT, keep_counts=[120 - 50, 0, 180 - 77])
+    assert np.array_equal(hi_k, 1 - lo_k)
+    # brute force on one sequence: the kept ones are exactly the K smallest
+    kept = np.flatnonzero(hi_k[:120])
+    assert set(kept.tolist()) == set(np.argsort(r[:120])[:50].tolist())
+    # protected tokens stay in both directions
+    hp = oc.select(r, cu, oc.THRESHOLD, tau=0.0, keep_first=3, keep_last=2, halt_high=True)   # everything above 0 halts
+    assert hp[:3].all() and hp[118:120].all() and hp[120:123].all() and hp[298:].all() and hp.sum() == 10
+
+
 def test_select_protected_prefix_suffix():
     r = np.float32([0.0, 0.0, 0.9, 0.8, 0.7, 0.6, 0.0, 0.0])
     cu = np.array([0, 8], dtype=np.int32)
@@ -373,6 +396,16 @@ def test_block_step_ffn_against_torch_restatement_and_closed_forms():
     assert np.allclose(oc.ffn_swiglu(-X, eye, eye, eye), 0.0, atol=1e-12)        # silu(-40) ~ -1.7e-16
     assert abs(oc.ffn_swiglu(np.array([[1.0]]), np.array([[1.0]]), np.array([[2.0]]), np.array([[3.0]]))[0, 0]
                - (1.0 / (1.0 + math.exp(-1.0))) * 2.0 * 3.0) < 1e-15
+    # block signal: the score is the change over the whole block; by the triangle inequality it lies within ||F|| / ||H|| of the
+    # attention score, and with a zero down projection the two signals coincide
+    rb = oc.block_step(H, W, w.cu, pos, sh, tau=tau, signal="block")
+    Hd = oc.f64(H)
+    want = np.linalg.norm(res["H1"] - Hd, axis=1) / np.linalg.norm(Hd, axis=1)
+    assert np.allclose(rb["r"], want.astype(np.float32), rtol=1e-6)
+    assert np.all(np.abs(rb["r"].astype(np.float64) - res["r"]) <= np.linalg.norm(res["F"], axis=1) / np.linalg.norm(Hd, axis=1) * (1 + 1e-6) + 1e-7)
+    assert np.array_equal(rb["mask"], oc.select(rb["r"], w.cu, oc.THRESHOLD, tau=tau))
+    Wz = dict(W); Wz["Wd"] = torch.zeros_like(W["Wd"])
+    assert np.array_equal(oc.block_step(H, Wz, w.cu, pos, sh, tau=tau, signal="block")["r"], res["r"])
     # row-sampled evaluation equals the full one on those rows
     r3 = oc.block_step(H, W, w.cu, pos, sh, attn_rows=[0, 77, 159])
     assert np.allclose(r3["H1"], res["H1"][[0, 77, 159]], rtol=1e-12, atol=1e-13)
