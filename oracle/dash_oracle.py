@@ -356,6 +356,34 @@ def block_step(H, weights: Dict[str, object], cu, pos, shape, norm_mode: int = R
     return out
 
 
+def decode_attention(q, Kc, Vc, cu, scale: Optional[float] = None):
+    """Attention of one new token per sequence over that sequence's cached keys and values (the decoding
+    stage, Preliminaries; halted prompt tokens have left the cache of the deeper layers, Appendix C "DASH
+    settings", so the packed cache simply holds fewer rows there).  No mask: the new token sees every cached
+    row of its sequence.  q [S,Hq,D]; Kc, Vc [n,Hkv,D] packed, cu int32 [S+1].  Returns (O [S,Hq,D], lse [S,Hq]);
+    an empty cache gives O = 0 and lse = -inf."""
+    q, Kc, Vc = f64(q), f64(Kc), f64(Vc)
+    cu = i32(cu)
+    S, Hq, D = q.shape
+    G = Hq // Kc.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    O = np.zeros((S, Hq, D))
+    lse = np.full((S, Hq), -np.inf)
+    for s in range(S):
+        a, b = int(cu[s]), int(cu[s + 1])
+        if b <= a:
+            continue
+        for h in range(Hq):
+            sc = (Kc[a:b, h // G] @ q[s, h]) * scale
+            mx = sc.max()
+            p = np.exp(sc - mx)
+            l = p.sum()
+            O[s, h] = (p / l) @ Vc[a:b, h // G]
+            lse[s, h] = mx + math.log(l)
+    return O, lse
+
+
 def kth_largest(r, k: int) -> float:
     """The k-th largest score (k >= 1): with tau set to it and the rule
     "halt iff r < tau", exactly k tokens stay when there are no ties."""

@@ -291,6 +291,41 @@ def test_attention_matches_library_sdpa():
 
 
 # ---------------------------------------------------------------------- glue
+def test_decode_attention_pins():
+    g = torch.Generator().manual_seed(21)
+    lengths = [37, 0, 5, 64]
+    cu = wl.cu_from_lengths(lengths).numpy()
+    n, Hq, Hkv, D = int(cu[-1]), 6, 2, 16
+    K = torch.randn(n, Hkv, D, generator=g, dtype=torch.float64)
+    V = torch.randn(n, Hkv, D, generator=g, dtype=torch.float64)
+    q = torch.randn(len(lengths), Hq, D, generator=g, dtype=torch.float64)
+    O, lse = oc.decode_attention(q, K, V, cu)
+    # library routine: torch SDPA without mask, one sequence at a time
+    for s, L in enumerate(lengths):
+        a = int(cu[s])
+        if L == 0:
+            assert not O[s].any() and np.isinf(lse[s]).all()
+            continue
+        k = K[a:a + L].transpose(0, 1).repeat_interleave(Hq // Hkv, 0)[None]
+        v = V[a:a + L].transpose(0, 1).repeat_interleave(Hq // Hkv, 0)[None]
+        ref = torch.nn.functional.scaled_dot_product_attention(q[s][None, :, None, :], k, v)[0, :, 0]
+        assert np.allclose(O[s], ref.numpy(), rtol=1e-10, atol=1e-12)
+    # the last prompt token's causal attention is a decode step over the whole prompt with its own query
+    Q = torch.randn(n, Hq, D, generator=g, dtype=torch.float64)
+    Oc, lc = oc.attention(Q, K, V, cu)
+    qs = torch.stack([Q[int(cu[s + 1]) - 1] if L else Q[0] for s, L in enumerate(lengths)])
+    Od, ld = oc.decode_attention(qs, K, V, cu)
+    for s, L in enumerate(lengths):
+        if L:
+            e = int(cu[s + 1]) - 1
+            assert np.allclose(Od[s], Oc[e], rtol=1e-12, atol=1e-14) and np.allclose(ld[s], lc[e], rtol=1e-12)
+    # closed forms: a single cached row returns its value; constant values return the constant; q = 0 the mean
+    O1, l1 = oc.decode_attention(q[:1], K[:1], V[:1], np.array([0, 1], dtype=np.int32))
+    assert np.allclose(O1[0], V[0].repeat_interleave(Hq // Hkv, 0).numpy())
+    Oz, lz = oc.decode_attention(torch.zeros_like(q[:1]), K[:37], V[:37], np.array([0, 37], dtype=np.int32))
+    assert np.allclose(Oz[0], V[:37].mean(0).repeat_interleave(Hq // Hkv, 0).numpy()) and np.allclose(lz, math.log(37))
+
+
 def test_rmsnorm_and_rope_properties():
     g = torch.Generator().manual_seed(10)
     H = torch.randn(9, 64, generator=g, dtype=torch.float64)
