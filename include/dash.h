@@ -187,6 +187,20 @@ int dash_varlen_attention(const void* Q, const void* K, const void* V, void* O, 
                           int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
                           void* ws, size_t ws_bytes, void* stream);
 
+/* ---- decoding stage: one new token per sequence over the packed KV cache ---
+ * (Preliminaries: decoding reuses the cached keys and values; Appendix C, "DASH settings":
+ * halting prompt tokens shortens the KV cache -- the cache of a deeper layer holds only the
+ * tokens that stayed active, i.e. the K and V rows a block step emits.)
+ * For sequence s and query head h:  out[s,h,:] = sum_j softmax_j(scale * q[s,h] . Kc[j,kv]) Vc[j,kv,:]
+ * over the cached rows cu[s] <= j < cu[s+1], kv = h / (Hq / Hkv); no mask.  An empty cache gives 0
+ * (lse = -inf).  q [S,Hq,D], out [S,Hq,D], Kc, Vc [n,Hkv,D], all DASH_BF16 (DASH_F32 is
+ * unsupported: the cache is read as stored), row strides ldq, ldo, ldk, ldv in elements.
+ * lse: NULL or fp32 [S,Hq].  Hq / Hkv <= 8; D in {64, 128}.  ws: dash_workspace_bytes(DASH_WS_DECODE). */
+int dash_decode_attention(const void* q, const void* Kc, const void* Vc, void* out, float* lse,
+                          int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                          const int32_t* cu_seqlens, int S, int64_t n, int Hq, int Hkv, int D, float scale,
+                          dash_dtype dt, void* ws, size_t ws_bytes, void* stream);
+
 /* ---- the whole block step (Alg. 1, loop body without the FFN) ------------ */
 typedef struct {
     int          d, Hq, Hkv, D;
@@ -203,6 +217,8 @@ typedef struct {
     const int32_t* keep_counts;    /* KEEP_COUNT: device int32 [S] */
     int          keep_first, keep_last;
     int          scatter_which;    /* rows of H~ written to x_full: 0 halted, 2 all */
+    void*        k_cache;          /* NULL, or [n, Hkv, D]: this block's keys (rotary applied) of the entering tokens, */
+    void*        v_cache;          /* and values: the rows a decoding step attends over at this depth (both or neither) */
 } dash_layer_cfg;
 
 /* Byte offsets of the intermediates inside the workspace of dash_layer_step
@@ -257,7 +273,7 @@ int dash_block_step(const dash_block_cfg* cfg, const void* H_in, const int32_t* 
                     void* ws, size_t ws_bytes, void* stream);
 
 /* ---- workspace sizes ------------------------------------------------------ */
-typedef enum { DASH_WS_SELECT = 0, DASH_WS_COMPACT = 1, DASH_WS_ATTENTION = 2 } dash_ws_op;
+typedef enum { DASH_WS_SELECT = 0, DASH_WS_COMPACT = 1, DASH_WS_ATTENTION = 2, DASH_WS_DECODE = 3 } dash_ws_op;
 /* n: rows allocated; S: sequences; Hq, Hkv, D, dt only matter for attention. */
 size_t dash_workspace_bytes(dash_ws_op op, int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt);
 

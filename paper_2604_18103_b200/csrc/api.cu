@@ -24,6 +24,7 @@ int* status_word_ptr() {
 size_t select_ws_bytes(int64_t n, int S);
 size_t compact_ws_bytes_pub(int64_t n);
 size_t attention_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt);
+size_t decode_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D);
 
 }  // namespace dash
 
@@ -82,6 +83,7 @@ extern "C" size_t dash_workspace_bytes(dash_ws_op op, int64_t n, int S, int Hq, 
         case DASH_WS_SELECT: return dash::select_ws_bytes(n, S);
         case DASH_WS_COMPACT: return dash::compact_ws_bytes_pub(n);
         case DASH_WS_ATTENTION: return dash::attention_ws_bytes(n, S, Hq, Hkv, D, dt);
+        case DASH_WS_DECODE: return dash::decode_ws_bytes(n, S, Hq, Hkv, D);
         default: return 0;
     }
 }

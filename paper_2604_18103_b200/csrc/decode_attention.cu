@@ -1,0 +1,429 @@
+// Decode-step attention: one new token per sequence attends over that sequence's packed KV cache
+// (the cache of the deeper layers holds only the tokens that stayed active; it simply has fewer rows).
+// HBM-bound: every cached key/value row is read once.  The G = Hq / Hkv query heads that share one KV
+// head form the (mostly empty) 128-row operand of the tcgen05 MMAs, so K and V tiles stream through
+// shared memory once per KV head; the keys of a sequence are split over persistent CTAs (flash-decoding),
+// whose partial (max, sum, O) results a small merge kernel combines.
+//   plan kernel   : items (sequence, KV head, key-block range), sized so that about four items exist per SM
+//   decode kernel : per item  S = Q K_j^T -> masked online softmax (one warp: the rows that exist) -> O += P V_j
+//   merge kernel  : O = sum_i 2^((m_i - m) c) O_i / sum_i 2^((m_i - m) c) l_i
+#include <math.h>
+
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace dash {
+
+using namespace ptx;
+
+constexpr int kDecBN = 128;                  // keys per block
+constexpr int kDecThreads = 64;              // warp 0: softmax (rows 0..31 of the tile, G of them real), warp 1: TMA + MMA issue
+constexpr int kDecRows = 8;                  // query heads per KV head the tile can hold (box of the Q load)
+constexpr long long kDecWaitCycles = 4000000000LL;
+constexpr uint32_t kDecTmemCols = 256;       // S | O
+
+struct DecItem { int s, kvh, b0, b1; };
+
+struct DecParams {
+    const int32_t* cu;
+    int S, Hq, Hkv, G;
+    float scale_log2, scale;
+    float* partial;             // [item][kDecRows][D + 2]: unnormalised O row, then m, l
+    const DecItem* plan;
+    const int* n_items;
+    unsigned int* ticket;
+    int* status;
+};
+
+// One CTA: per sequence the number of key blocks, a common chunk length (blocks per item) so that about
+// `target` items exist, then the items of every (sequence, KV head) written next to each other.
+__global__ void __launch_bounds__(256)
+decode_plan_kernel(const int32_t* __restrict__ cu, int S, int Hkv, int target, DecItem* __restrict__ plan, int2* __restrict__ seg,
+                   int* __restrict__ n_items, unsigned int* __restrict__ ticket, int max_items) {
+    __shared__ long long s_total;
+    __shared__ int s_chunk;
+    if (threadIdx.x == 0) s_total = 0;
+    __syncthreads();
+    long long mine = 0;
+    for (int s = threadIdx.x; s < S; s += blockDim.x) mine += (cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN;
+    atomicAdd((unsigned long long*)&s_total, (unsigned long long)mine);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const long long all = s_total * Hkv;
+        long long chunk = (all + target - 1) / target;
+        s_chunk = (int)(chunk < 1 ? 1 : chunk);
+        // items of (s, kvh) are contiguous; a serial walk is a few thousand steps at most
+        int k = 0;
+        for (int s = 0; s < S; ++s) {
+            const int nb = (cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN;
+            for (int h = 0; h < Hkv; ++h) {
+                const int first = k;
+                for (int b = 0; b < nb && k < max_items; b += s_chunk) {
+                    DecItem it = {s, h, b, min(b + s_chunk, nb)};
+                    plan[k++] = it;
+                }
+                seg[s * Hkv + h] = make_int2(first, k - first);
+            }
+        }
+        *n_items = k;
+        *ticket = 0u;
+    }
+}
+
+template <int D>
+struct DecSmem {
+    static constexpr int kTileBytes = kDecBN * D * 2;
+    static constexpr int kQ = 0, kK = kTileBytes, kV = 2 * kTileBytes, kBars = 3 * kTileBytes;
+    static constexpr int kTotal = kBars + 128;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kDecThreads)
+decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+              const __grid_constant__ CUtensorMap mapV, const DecParams p, int q_box_heads) {
+    extern __shared__ uint8_t smem_raw[];
+    using L = DecSmem<D>;
+    constexpr int KCH = D / 64;
+    constexpr int kChunkBytes = kDecBN * 128;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base + L::kQ, sK = smem_base + L::kK, sV = smem_base + L::kV;
+    const uint32_t bars = smem_base + L::kBars;
+    const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_o = bars + 32, bar_p0 = bars + 40, bar_p1 = bars + 48;
+    const uint32_t tmem_slot = bars + 64;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 64);
+    volatile uint32_t* abort_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 68);
+    volatile int* item_gen = reinterpret_cast<volatile int*>(smem_gen + L::kBars + 72);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // rows of the Q tile that no load ever writes must not hold NaN patterns: clear the tile once
+    for (int i = tid * 16; i < L::kTileBytes; i += kDecThreads * 16) *reinterpret_cast<uint4*>(smem_gen + L::kQ + i) = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+    if (warp == 1) {
+        if (lane == 0) {
+            mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1);
+            mbar_init(bar_s, 1); mbar_init(bar_o, 1); mbar_init(bar_p0, 32); mbar_init(bar_p1, 32);
+            *abort_gen = 0;
+            fence_barrier_init();
+            fence_proxy_async_smem();
+            prefetch_tensormap(&mapQ); prefetch_tensormap(&mapK); prefetch_tensormap(&mapV);
+        }
+        __syncwarp();
+        tmem_alloc(tmem_slot, kDecTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot_gen;
+    const uint32_t tS = tmem, tP = tmem, tO = tmem + 128;
+    constexpr uint32_t idesc_s = idesc_bf16_f32(128, kDecBN, false, false);
+    constexpr uint32_t idesc_o = idesc_bf16_f32(128, D, false, true);
+    const int n_items = *p.n_items;
+    uint32_t blk0 = 0, items_done = 0;       // barrier phases run on across the items of this CTA
+
+    for (;;) {
+        if (tid == 0) *item_gen = (int)atomicAdd(p.ticket, 1u);
+        __syncthreads();
+        const int item = *item_gen;
+        if (item >= n_items || *abort_gen) break;
+        tc_fence_after();
+        const DecItem it = p.plan[item];
+        const int seq_a = p.cu[it.s], len = p.cu[it.s + 1] - seq_a;
+        const int nblk = it.b1 - it.b0;
+        const int last_blk = (len + kDecBN - 1) / kDecBN - 1;       // the block of the sequence with a ragged end
+        if (warp == 1) {
+            if (lane == 0) {
+                bool ok = true;
+                mbar_arrive_expect_tx(bar_q, (uint32_t)(KCH * q_box_heads * 128));
+                for (int c = 0; c < KCH; ++c) tma_load_3d(sQ + c * kChunkBytes, &mapQ, bar_q, c * 64, it.kvh * p.G, it.s);
+                mbar_arrive_expect_tx(bar_k, L::kTileBytes);
+                for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, it.kvh, seq_a + it.b0 * kDecBN);
+                mbar_arrive_expect_tx(bar_v, L::kTileBytes);
+                for (int c = 0; c < KCH; ++c) tma_load_3d(sV + c * kChunkBytes, &mapV, bar_v, c * 64, it.kvh, seq_a + it.b0 * kDecBN);
+                auto issue_s = [&]() {
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = (kk >> 2) * kChunkBytes + (kk & 3) * 32;
+                        mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), idesc_s, kk > 0);
+                    }
+                    tc_commit(bar_s);
+                };
+                ok = mbar_wait(bar_q, items_done & 1, kDecWaitCycles) && mbar_wait(bar_k, blk0 & 1, kDecWaitCycles);
+                if (ok) issue_s();
+                for (int j = 0; j < nblk && ok; ++j) {
+                    const uint32_t ph = (blk0 + j) & 1;
+                    ok = mbar_wait(bar_s, ph, kDecWaitCycles);               // S_j done: the K buffer is free
+                    if (!ok) break;
+                    if (j + 1 < nblk) {
+                        mbar_arrive_expect_tx(bar_k, L::kTileBytes);
+                        for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, it.kvh, seq_a + (it.b0 + j + 1) * kDecBN);
+                    }
+                    ok = mbar_wait(bar_p0, ph, kDecWaitCycles) && mbar_wait(bar_v, ph, kDecWaitCycles);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < kDecBN / 32; ++kk)
+                        mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
+                    ok = mbar_wait(bar_p1, ph, kDecWaitCycles);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = kDecBN / 32; kk < kDecBN / 16; ++kk)
+                        mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, 1);
+                    tc_commit(bar_o);
+                    if (j + 1 < nblk) {
+                        ok = mbar_wait(bar_k, (blk0 + j + 1) & 1, kDecWaitCycles);
+                        if (!ok) break;
+                        issue_s();                                         // in issue order behind PV_j, which reads P_j from the same columns
+                    }
+                    ok = mbar_wait(bar_o, ph, kDecWaitCycles);              // PV_j done: the V buffer is free
+                    if (!ok) break;
+                    if (j + 1 < nblk) {
+                        mbar_arrive_expect_tx(bar_v, L::kTileBytes);
+                        for (int c = 0; c < KCH; ++c) tma_load_3d(sV + c * kChunkBytes, &mapV, bar_v, c * 64, it.kvh, seq_a + (it.b0 + j + 1) * kDecBN);
+                    }
+                }
+                if (!ok) { *abort_gen = 1; atomicExch(p.status, DASH_ERR_TIMEOUT); }
+            }
+        } else {
+            // ---- softmax warp: lane <-> row of the tile = query head kvh * G + lane (lanes >= G compute on zeros) ----
+            float m = -INFINITY, l = 0.f;
+            bool ok = true;
+            for (int j = 0; j < nblk; ++j) {
+                const uint32_t ph = (blk0 + j) & 1;
+                ok = mbar_wait(bar_s, ph, kDecWaitCycles);
+                if (!ok || *abort_gen) { ok = false; break; }
+                tc_fence_after();
+                uint32_t sreg[128];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, &sreg[c * 32]);
+                tmem_wait_ld();
+                const bool ragged = (it.b0 + j == last_blk);
+                const int valid = len - (it.b0 + j) * kDecBN;               // keys of this block that exist (>= 1)
+                if (ragged) {
+#pragma unroll
+                    for (int c = 0; c < 128; ++c)
+                        if (c >= valid) sreg[c] = 0xff800000u;             // -inf: past the end of the sequence's cache
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 128; c += 8) {
+                    mx0 = fmax3(mx0, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+                    mx2 = fmax3(mx2, __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
+                    mx3 = fmax3(mx3, __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
+                }
+                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                // the reference max only moves when the block max exceeds it by more than 2^8 (then O is rescaled)
+                const bool grow = (mx - m) * p.scale_log2 > 8.0f;
+                const float m_new = grow ? mx : m;
+                const float msl = m_new * p.scale_log2;
+                const float alpha = grow ? ex2((m - m_new) * p.scale_log2) : 1.0f;
+                if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                    ok = mbar_wait(bar_o, (blk0 + j - 1) & 1, kDecWaitCycles);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c = 0; c < D / 8; ++c) {
+                        uint32_t o[8];
+                        tmem_ld8(tO + c * 8, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tmem_st8(tO + c * 8, o);
+                    }
+                }
+                if (ragged) {
+                    // cached rows past the end of the sequence may hold anything: zero them (0 * garbage must not make a NaN)
+                    ok = mbar_wait(bar_v, ph, kDecWaitCycles);
+                    if (!ok) break;
+                    for (int r = lane; r < kDecBN; r += 32) {
+                        if (r >= valid) {
+#pragma unroll
+                            for (int c = 0; c < KCH; ++c) {
+                                uint4* rowp = reinterpret_cast<uint4*>(smem_gen + L::kV + c * kChunkBytes + r * 128);
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) rowp[e] = make_uint4(0, 0, 0, 0);
+                            }
+                        }
+                    }
+                    fence_proxy_async_smem();
+                }
+                float2 sumA = make_float2(0.f, 0.f), sumB = make_float2(0.f, 0.f);
+                const float2 sl2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-msl, -msl);
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                    for (int c = half * 64; c < half * 64 + 64; c += 4) {
+                        const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), sl2, nm2);
+                        const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), sl2, nm2);
+                        float2 pa, pb;
+                        pa.x = ex2(xa.x); pa.y = ex2(xa.y); pb.x = ex2(xb.x); pb.y = ex2(xb.y);
+                        sumA = __fadd2_rn(sumA, pa);
+                        sumB = __fadd2_rn(sumB, pb);
+                        sreg[c >> 1] = pack_bf16(pa.x, pa.y);
+                        sreg[(c >> 1) + 1] = pack_bf16(pb.x, pb.y);
+                    }
+                    tmem_st32(tP + half * 32, &sreg[half * 32]);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(half == 0 ? bar_p0 : bar_p1);
+                }
+                l = l * alpha + ((sumA.x + sumA.y) + (sumB.x + sumB.y));
+                m = m_new;
+            }
+            if (ok) ok = mbar_wait(bar_o, (blk0 + nblk - 1) & 1, kDecWaitCycles);
+            if (ok && !*abort_gen) {
+                tc_fence_after();
+                float* dst = p.partial + ((size_t)item * kDecRows + lane) * (D + 2);
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_wait_ld();
+                    if (lane < p.G) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2)
+                            *reinterpret_cast<float2*>(dst + c * 32 + e) = make_float2(__uint_as_float(o[e]), __uint_as_float(o[e + 1]));
+                    }
+                }
+                if (lane < p.G) { dst[D] = m; dst[D + 1] = l; }
+            } else if (!ok && lane == 0) {
+                *abort_gen = 1;
+                atomicExch(p.status, DASH_ERR_TIMEOUT);
+            }
+        }
+        tc_fence_before();
+        __syncthreads();                      // end of the item: O read out, every tile buffer free
+        blk0 += (uint32_t)nblk;
+        ++items_done;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kDecTmemCols);
+    }
+}
+
+// One CTA per (sequence, query head): combine the partial results of the key splits.
+template <bool OUT_F32>
+__global__ void __launch_bounds__(128)
+decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ seg, const int* __restrict__ n_items, int Hq, int G, int D,
+                    float scale_log2, float scale, void* __restrict__ out, int64_t ldo, float* __restrict__ lse) {
+    const int s = blockIdx.x / Hq, h = blockIdx.x % Hq;
+    const int kvh = h / G, row = h % G, Hkv = Hq / G;
+    int2 sg = seg[s * Hkv + kvh];
+    if (sg.x + sg.y > *n_items) sg.y = max(0, *n_items - sg.x);
+    float mall = -INFINITY;
+    for (int i = 0; i < sg.y; ++i) mall = fmaxf(mall, partial[((size_t)(sg.x + i) * kDecRows + row) * (D + 2) + D]);
+    float lall = 0.f;
+    for (int i = 0; i < sg.y; ++i) {
+        const float* pp = partial + ((size_t)(sg.x + i) * kDecRows + row) * (D + 2);
+        lall += pp[D + 1] * exp2f((pp[D] - mall) * scale_log2);
+    }
+    for (int c = threadIdx.x; c < D; c += blockDim.x) {
+        float acc = 0.f;
+        for (int i = 0; i < sg.y; ++i) {
+            const float* pp = partial + ((size_t)(sg.x + i) * kDecRows + row) * (D + 2);
+            acc += pp[c] * exp2f((pp[D] - mall) * scale_log2);
+        }
+        const float v = sg.y > 0 ? acc / lall : 0.f;
+        if (OUT_F32) reinterpret_cast<float*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = v;
+        else reinterpret_cast<__nv_bfloat16*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = __float2bfloat16(v);
+    }
+    if (lse && threadIdx.x == 0) lse[(int64_t)s * Hq + h] = sg.y > 0 ? mall * scale + logf(lall) : -INFINITY;
+}
+
+static int decode_max_items(int S, int Hkv) { return 4 * sm_count() + S * Hkv; }
+
+size_t decode_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D) {
+    (void)n; (void)Hq;
+    const size_t items = (size_t)decode_max_items(S, Hkv);
+    return 256 + align_up(items * sizeof(DecItem), 256) + align_up((size_t)S * Hkv * sizeof(int2), 256) +
+           align_up(items * kDecRows * (size_t)(D + 2) * sizeof(float), 256);
+}
+
+// bf16 tensor [rows, heads, D]: box = 64 x box_heads x box_rows, 128-byte swizzle
+static int make_map_heads_box(CUtensorMap* map, const void* base, int64_t rows, int heads, int D, int64_t ld, int box_heads, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return DASH_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)heads, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)ld * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DASH_OK : DASH_ERR_CUDA;
+}
+
+template <int D>
+static int launch_decode(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const DecParams& p, int box_heads, int grid,
+                         cudaStream_t st) {
+    using L = DecSmem<D>;
+    const int smem = L::kTotal + 1024;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
+        configured = true;
+    }
+    decode_kernel<D><<<grid, kDecThreads, smem, st>>>(mq, mk, mv, p, box_heads);
+    return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+}
+
+}  // namespace dash
+
+using namespace dash;
+
+extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* Vc, void* out, float* lse,
+                                     int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                                     const int32_t* cu_seqlens, int S, int64_t n, int Hq, int Hkv, int D, float scale,
+                                     dash_dtype dt, void* ws, size_t ws_bytes, void* stream) {
+    if (n < 0 || S < 1 || Hq < 1 || Hkv < 1 || !cu_seqlens) return DASH_ERR_INVALID_ARG;
+    if (dt != DASH_F32 && dt != DASH_BF16) return DASH_ERR_INVALID_ARG;
+    if (dt != DASH_BF16) return DASH_ERR_UNSUPPORTED;                 // the cache is read as stored: bf16 only
+    if (D != 64 && D != 128) return DASH_ERR_UNSUPPORTED;
+    if (Hq % Hkv) return DASH_ERR_INVALID_ARG;
+    const int G = Hq / Hkv;
+    if (G > kDecRows) return DASH_ERR_UNSUPPORTED;
+    if (n > 0x7fffffffLL || S > 0x7fffffff / Hq) return DASH_ERR_INVALID_ARG;
+    if (!q || !out || (n > 0 && (!Kc || !Vc))) return DASH_ERR_INVALID_ARG;
+    if (ldq < (int64_t)Hq * D || ldo < (int64_t)Hq * D || ldk < (int64_t)Hkv * D || ldv < (int64_t)Hkv * D) return DASH_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || (n > 0 && (!aligned16(Kc) || !aligned16(Vc)))) return DASH_ERR_INVALID_ARG;
+    if ((ldq * 2) % 16 || (ldk * 2) % 16 || (ldv * 2) % 16 || (ldo * 2) % 16) return DASH_ERR_INVALID_ARG;
+    if (!(scale > 0.f)) return DASH_ERR_INVALID_ARG;
+    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < decode_ws_bytes(n, S, Hq, Hkv, D)) return DASH_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int max_items = decode_max_items(S, Hkv);
+    char* w = (char*)ws;
+    DecItem* plan = (DecItem*)(w + 256);
+    int2* seg = (int2*)(w + 256 + align_up((size_t)max_items * sizeof(DecItem), 256));
+    float* partial = (float*)((char*)seg + align_up((size_t)S * Hkv * sizeof(int2), 256));
+    decode_plan_kernel<<<1, 256, 0, st>>>(cu_seqlens, S, Hkv, 4 * sm_count(), plan, seg, (int*)(w + 4), (unsigned int*)w, max_items);
+    DASH_CUDA_TRY(cudaGetLastError());
+    const float scale_log2 = scale * 1.4426950408889634f;
+    if (n > 0) {
+        CUtensorMap mq, mk, mv;
+        int rc;
+        const int box_heads = Hq < kDecRows ? Hq : kDecRows;
+        if ((rc = make_map_heads_box(&mq, q, S, Hq, D, ldq, box_heads, 1)) != DASH_OK) return rc;
+        if ((rc = make_map_heads_box(&mk, Kc, n, Hkv, D, ldk, 1, kDecBN)) != DASH_OK) return rc;
+        if ((rc = make_map_heads_box(&mv, Vc, n, Hkv, D, ldv, 1, kDecBN)) != DASH_OK) return rc;
+        DecParams p;
+        p.cu = cu_seqlens; p.S = S; p.Hq = Hq; p.Hkv = Hkv; p.G = G;
+        p.scale = scale; p.scale_log2 = scale_log2;
+        p.partial = partial; p.plan = plan; p.n_items = (const int*)(w + 4); p.ticket = (unsigned int*)w;
+        p.status = status_word_ptr();
+        if (!p.status) return DASH_ERR_CUDA;
+        int grid = 2 * sm_count();
+        if (grid > max_items) grid = max_items;
+        rc = D == 128 ? launch_decode<128>(mq, mk, mv, p, box_heads, grid, st) : launch_decode<64>(mq, mk, mv, p, box_heads, grid, st);
+        if (rc != DASH_OK) return rc;
+    }
+    decode_merge_kernel<false><<<S * Hq, 128, 0, st>>>(partial, seg, (const int*)(w + 4), Hq, G, D, scale_log2, scale, out, ldo, lse);
+    DASH_CUDA_TRY(cudaGetLastError());
+    return DASH_OK;
+}

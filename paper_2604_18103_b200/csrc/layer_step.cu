@@ -218,6 +218,7 @@ static bool cfg_ok(const dash_layer_cfg* c) {
     if (c->keep_first < 0 || c->keep_last < 0) return false;
     if (c->scatter_which != 0 && c->scatter_which != 2) return false;
     if (!(c->rope_base > 0.0)) return false;
+    if ((c->k_cache == nullptr) != (c->v_cache == nullptr)) return false;
     return true;
 }
 
@@ -296,6 +297,12 @@ static int attention_branch(const dash_layer_cfg* cfg, const void* H_in, const i
     else if (D == 128) rope_kernel<false, 128><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
     else rope_kernel<false, 64><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
     DASH_CUDA_TRY(cudaGetLastError());
+    if (cfg->k_cache) {
+        // this depth's KV cache rows: keys (rotary applied) and values of the entering tokens, packed [n, Hkv, D]
+        const int64_t kvb = (int64_t)Hkv * D * es;
+        if ((rc = dash_scatter(W.QKV + (int64_t)Hq * D * es, n, kvb, nq * es, nullptr, nullptr, 2, n_dev, cfg->k_cache, kvb, st)) != DASH_OK) return rc;
+        if ((rc = dash_scatter(W.QKV + (int64_t)(Hq + Hkv) * D * es, n, kvb, nq * es, nullptr, nullptr, 2, n_dev, cfg->v_cache, kvb, st)) != DASH_OK) return rc;
+    }
     // attention over the packed active set
     rc = dash_varlen_attention(W.QKV, W.QKV + (int64_t)Hq * D * es, W.QKV + (int64_t)(Hq + Hkv) * D * es, W.O, nullptr, nq, nq, nq,
                                (int64_t)Hq * D, cu_in, S, n, max_seqlen, Hq, Hkv, D, 1.0f / sqrtf((float)D), 1, cfg->dt,

@@ -19,7 +19,7 @@ F32, BF16 = 0, 1
 NORM_REL, NORM_ABS = 0, 1
 SEL_THRESHOLD, SEL_KEEP_COUNT, SEL_THRESHOLD_HALT_HIGH, SEL_KEEP_COUNT_HALT_HIGH = 0, 1, 2, 3
 SIGNAL_ATTN, SIGNAL_BLOCK = 0, 1
-WS_SELECT, WS_COMPACT, WS_ATTENTION = 0, 1, 2
+WS_SELECT, WS_COMPACT, WS_ATTENTION, WS_DECODE = 0, 1, 2, 3
 OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -29,7 +29,7 @@ EXPORTS = [
     "dash_status_string", "dash_check_status", "dash_keep_count", "dash_flops_per_layer", "dash_flops_speedup",
     "dash_delta_norm", "dash_select", "dash_compact", "dash_scatter", "dash_varlen_attention",
     "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes", "dash_compact_static",
-    "dash_block_workspace", "dash_block_step",
+    "dash_block_workspace", "dash_block_step", "dash_decode_attention",
 ]
 COMPACT_STATIC_MAX_ROWS = 1 << 20
 
@@ -49,7 +49,7 @@ class LayerCfg(Structure):
                 ("Wqkv", c_void_p), ("Wo", c_void_p), ("rms_weight", c_void_p), ("rms_eps", c_float),
                 ("rope_base", c_double), ("norm_mode", c_int), ("norm_eps", c_float), ("sel_mode", c_int),
                 ("tau", c_float), ("keep_counts", c_void_p), ("keep_first", c_int), ("keep_last", c_int),
-                ("scatter_which", c_int)]
+                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p)]
 
 
 class LayerWsLayout(Structure):
@@ -102,6 +102,8 @@ def lib() -> ctypes.CDLL:
         L.dash_layer_step.argtypes = [POINTER(LayerCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_size_t, c_void_p]
+        L.dash_decode_attention.argtypes = [c_void_p] * 5 + [c_int64] * 4 + [c_void_p, c_int, c_int64, c_int, c_int, c_int, c_float, c_int,
+                                                                          c_void_p, c_size_t, c_void_p]
         L.dash_block_workspace.argtypes = [POINTER(BlockCfg), c_int64, c_int, POINTER(BlockWsLayout)]
         L.dash_block_step.argtypes = [POINTER(BlockCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -279,6 +281,26 @@ def dash_varlen_attention(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, cu_
     return (O, lse) if want_lse else O
 
 
+def dash_decode_attention(q: torch.Tensor, Kc: torch.Tensor, Vc: torch.Tensor, cu_seqlens: torch.Tensor, scale: Optional[float] = None,
+                          out: Optional[torch.Tensor] = None, want_lse: bool = False, ws: Optional[torch.Tensor] = None):
+    """q [S,Hq,D] (one new token per sequence), Kc, Vc [n,Hkv,D] packed caches.  Returns out [S,Hq,D] (and lse [S,Hq])."""
+    _dev(q, Kc, Vc, cu_seqlens)
+    S, Hq, D = q.shape
+    n, Hkv = Kc.shape[0], Kc.shape[1]
+    if scale is None:
+        scale = 1.0 / (D ** 0.5)
+    if out is None:
+        out = torch.empty(S, Hq, D, dtype=q.dtype, device=q.device)
+    lse = torch.empty(S, Hq, dtype=torch.float32, device=q.device) if want_lse else None
+    if ws is None:
+        ws = workspace(dash_workspace_bytes(WS_DECODE, n, S, Hq, Hkv, D, dtype_code(q)), q.device)
+    st = lib().dash_decode_attention(_p(q), _p(Kc), _p(Vc), _p(out), _p(lse), q.stride(0), Kc.stride(0) if n else Hkv * D,
+                                     Vc.stride(0) if n else Hkv * D, out.stride(0), _p(cu_seqlens), S, n, Hq, Hkv, D, float(scale),
+                                     dtype_code(q), _p(ws), ws.numel(), _stream())
+    _check(st, "dash_decode_attention")
+    return (out, lse) if want_lse else out
+
+
 # ---- the block step ---------------------------------------------------------------
 class Layer:
     """Device-resident weights and configuration of one block for dash_layer_step."""
@@ -292,10 +314,16 @@ class Layer:
         self.keep_counts = keep_counts
         self.cfg = LayerCfg(shape.d, shape.Hq, shape.Hkv, shape.D, dtype_code(self.Wo), self.Wqkv.data_ptr(), self.Wo.data_ptr(),
                             self.rms_w.data_ptr(), shape.rms_eps, shape.rope_base, norm_mode, norm_eps, sel_mode, tau,
-                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which)
+                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None)
 
     def set_tau(self, tau: float):
         self.cfg.tau = float(tau)
+
+    def set_kv_cache(self, k_cache: Optional[torch.Tensor], v_cache: Optional[torch.Tensor]):
+        """[n, Hkv, D] buffers that receive this block's keys (rotary applied) and values, or None."""
+        self.k_cache, self.v_cache = k_cache, v_cache
+        self.cfg.k_cache = k_cache.data_ptr() if k_cache is not None else None
+        self.cfg.v_cache = v_cache.data_ptr() if v_cache is not None else None
 
 
 def dash_layer_workspace(layer: Layer, n: int, S: int) -> LayerWsLayout:
@@ -327,6 +355,12 @@ class Block:
 
     def set_tau(self, tau: float):
         self.cfg.attn.tau = float(tau)
+
+    def set_kv_cache(self, k_cache: Optional[torch.Tensor], v_cache: Optional[torch.Tensor]):
+        """[n, Hkv, D] buffers that receive this block's keys (rotary applied) and values, or None."""
+        self.k_cache, self.v_cache = k_cache, v_cache
+        self.cfg.attn.k_cache = k_cache.data_ptr() if k_cache is not None else None
+        self.cfg.attn.v_cache = v_cache.data_ptr() if v_cache is not None else None
 
     def set_keep_counts(self, keep_counts: Optional[torch.Tensor], sel_mode: int):
         self.keep_counts = keep_counts
