@@ -39,34 +39,42 @@ struct DecParams {
 // `target` items exist, then the items of every (sequence, KV head) written next to each other.
 __global__ void __launch_bounds__(256)
 decode_plan_kernel(const int32_t* __restrict__ cu, int S, int Hkv, int target, DecItem* __restrict__ plan, int2* __restrict__ seg,
-                   int* __restrict__ n_items, unsigned int* __restrict__ ticket, int max_items) {
-    __shared__ long long s_total;
+                   int* __restrict__ n_items, unsigned int* __restrict__ ticket, int max_items, int* __restrict__ seq_first) {
+    __shared__ unsigned long long s_total;
     __shared__ int s_chunk;
     if (threadIdx.x == 0) s_total = 0;
     __syncthreads();
-    long long mine = 0;
-    for (int s = threadIdx.x; s < S; s += blockDim.x) mine += (cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN;
-    atomicAdd((unsigned long long*)&s_total, (unsigned long long)mine);
+    unsigned long long mine = 0;
+    for (int s = threadIdx.x; s < S; s += blockDim.x) mine += (unsigned long long)((cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN);
+    atomicAdd(&s_total, mine);
     __syncthreads();
     if (threadIdx.x == 0) {
-        const long long all = s_total * Hkv;
-        long long chunk = (all + target - 1) / target;
+        const long long all = (long long)s_total * Hkv;
+        const long long chunk = (all + target - 1) / target;
         s_chunk = (int)(chunk < 1 ? 1 : chunk);
-        // items of (s, kvh) are contiguous; a serial walk is a few thousand steps at most
+        // first item of every sequence (its Hkv heads follow each other): one short serial pass over the sequences
         int k = 0;
         for (int s = 0; s < S; ++s) {
+            seq_first[s] = k;
             const int nb = (cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN;
-            for (int h = 0; h < Hkv; ++h) {
-                const int first = k;
-                for (int b = 0; b < nb && k < max_items; b += s_chunk) {
-                    DecItem it = {s, h, b, min(b + s_chunk, nb)};
-                    plan[k++] = it;
-                }
-                seg[s * Hkv + h] = make_int2(first, k - first);
-            }
+            k += ((nb + s_chunk - 1) / s_chunk) * Hkv;
         }
-        *n_items = k;
+        *n_items = k < max_items ? k : max_items;
         *ticket = 0u;
+    }
+    __syncthreads();
+    const int chunk = s_chunk;
+    for (int sh = threadIdx.x; sh < S * Hkv; sh += blockDim.x) {
+        const int s = sh / Hkv, h = sh % Hkv;
+        const int nb = (cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN;
+        const int per = (nb + chunk - 1) / chunk;
+        const int first = seq_first[s] + h * per;
+        int cnt = 0;
+        for (int i = 0; i < per && first + i < max_items; ++i, ++cnt) {
+            DecItem it = {s, h, i * chunk, min((i + 1) * chunk, nb)};
+            plan[first + i] = it;
+        }
+        seg[sh] = make_int2(first, cnt);
     }
 }
 
@@ -308,33 +316,55 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     }
 }
 
-// One CTA per (sequence, query head): combine the partial results of the key splits.
+// One CTA per (sequence, query head): combine the partial results of the key splits.  The weights of the splits are formed
+// in parallel over the splits, then every thread sums its column over them (independent loads).
+constexpr int kMergeMaxSplits = 1024;
 template <bool OUT_F32>
 __global__ void __launch_bounds__(128)
-decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ seg, const int* __restrict__ n_items, int Hq, int G, int D,
+decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ seg, int Hq, int G, int D,
                     float scale_log2, float scale, void* __restrict__ out, int64_t ldo, float* __restrict__ lse) {
+    __shared__ float s_w[kMergeMaxSplits];
+    __shared__ float s_red[4];
+    __shared__ float s_m, s_l;
     const int s = blockIdx.x / Hq, h = blockIdx.x % Hq;
     const int kvh = h / G, row = h % G, Hkv = Hq / G;
-    int2 sg = seg[s * Hkv + kvh];
-    if (sg.x + sg.y > *n_items) sg.y = max(0, *n_items - sg.x);
-    float mall = -INFINITY;
-    for (int i = 0; i < sg.y; ++i) mall = fmaxf(mall, partial[((size_t)(sg.x + i) * kDecRows + row) * (D + 2) + D]);
-    float lall = 0.f;
-    for (int i = 0; i < sg.y; ++i) {
-        const float* pp = partial + ((size_t)(sg.x + i) * kDecRows + row) * (D + 2);
-        lall += pp[D + 1] * exp2f((pp[D] - mall) * scale_log2);
+    const int2 sg = seg[s * Hkv + kvh];
+    const int cnt = sg.y < kMergeMaxSplits ? sg.y : kMergeMaxSplits;
+    const size_t stride = (size_t)kDecRows * (D + 2);
+    const float* base = partial + ((size_t)sg.x * kDecRows + row) * (D + 2);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    float mx = -INFINITY;
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) mx = fmaxf(mx, base[i * stride + D]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) s_red[w] = mx;
+    __syncthreads();
+    if (threadIdx.x == 0) s_m = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+    __syncthreads();
+    const float mall = s_m;
+    float ls = 0.f;
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+        const float wi = exp2f((base[i * stride + D] - mall) * scale_log2);
+        s_w[i] = wi;
+        ls += wi * base[i * stride + D + 1];
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+    __syncthreads();
+    if (lane == 0) s_red[w] = ls;
+    __syncthreads();
+    if (threadIdx.x == 0) s_l = (s_red[0] + s_red[1]) + (s_red[2] + s_red[3]);
+    __syncthreads();
+    const float lall = s_l;
     for (int c = threadIdx.x; c < D; c += blockDim.x) {
         float acc = 0.f;
-        for (int i = 0; i < sg.y; ++i) {
-            const float* pp = partial + ((size_t)(sg.x + i) * kDecRows + row) * (D + 2);
-            acc += pp[c] * exp2f((pp[D] - mall) * scale_log2);
-        }
-        const float v = sg.y > 0 ? acc / lall : 0.f;
+#pragma unroll 8
+        for (int i = 0; i < cnt; ++i) acc += s_w[i] * base[i * stride + c];
+        const float v = cnt > 0 ? acc / lall : 0.f;
         if (OUT_F32) reinterpret_cast<float*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = v;
         else reinterpret_cast<__nv_bfloat16*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = __float2bfloat16(v);
     }
-    if (lse && threadIdx.x == 0) lse[(int64_t)s * Hq + h] = sg.y > 0 ? mall * scale + logf(lall) : -INFINITY;
+    if (lse && threadIdx.x == 0) lse[(int64_t)s * Hq + h] = cnt > 0 ? mall * scale + logf(lall) : -INFINITY;
 }
 
 static int decode_max_items(int S, int Hkv) { return 4 * sm_count() + S * Hkv; }
@@ -342,7 +372,7 @@ static int decode_max_items(int S, int Hkv) { return 4 * sm_count() + S * Hkv; }
 size_t decode_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D) {
     (void)n; (void)Hq;
     const size_t items = (size_t)decode_max_items(S, Hkv);
-    return 256 + align_up(items * sizeof(DecItem), 256) + align_up((size_t)S * Hkv * sizeof(int2), 256) +
+    return 256 + align_up(items * sizeof(DecItem), 256) + align_up((size_t)S * Hkv * sizeof(int2), 256) + align_up((size_t)S * sizeof(int), 256) +
            align_up(items * kDecRows * (size_t)(D + 2) * sizeof(float), 256);
 }
 
@@ -401,8 +431,9 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
     char* w = (char*)ws;
     DecItem* plan = (DecItem*)(w + 256);
     int2* seg = (int2*)(w + 256 + align_up((size_t)max_items * sizeof(DecItem), 256));
-    float* partial = (float*)((char*)seg + align_up((size_t)S * Hkv * sizeof(int2), 256));
-    decode_plan_kernel<<<1, 256, 0, st>>>(cu_seqlens, S, Hkv, 4 * sm_count(), plan, seg, (int*)(w + 4), (unsigned int*)w, max_items);
+    int* seq_first = (int*)((char*)seg + align_up((size_t)S * Hkv * sizeof(int2), 256));
+    float* partial = (float*)((char*)seq_first + align_up((size_t)S * sizeof(int), 256));
+    decode_plan_kernel<<<1, 256, 0, st>>>(cu_seqlens, S, Hkv, 4 * sm_count(), plan, seg, (int*)(w + 4), (unsigned int*)w, max_items, seq_first);
     DASH_CUDA_TRY(cudaGetLastError());
     const float scale_log2 = scale * 1.4426950408889634f;
     if (n > 0) {
@@ -423,7 +454,7 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
         rc = D == 128 ? launch_decode<128>(mq, mk, mv, p, box_heads, grid, st) : launch_decode<64>(mq, mk, mv, p, box_heads, grid, st);
         if (rc != DASH_OK) return rc;
     }
-    decode_merge_kernel<false><<<S * Hq, 128, 0, st>>>(partial, seg, (const int*)(w + 4), Hq, G, D, scale_log2, scale, out, ldo, lse);
+    decode_merge_kernel<false><<<S * Hq, 128, 0, st>>>(partial, seg, Hq, G, D, scale_log2, scale, out, ldo, lse);
     DASH_CUDA_TRY(cudaGetLastError());
     return DASH_OK;
 }
