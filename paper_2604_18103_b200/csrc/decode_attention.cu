@@ -29,11 +29,48 @@ struct DecParams {
     int S, Hq, Hkv, G;
     float scale_log2, scale;
     float* partial;             // [item][kDecRows][D + 2]: unnormalised O row, then m, l
-    const DecItem* plan;
+    const DecItem* plan;        // null: the CTAs plan for themselves (S <= kSelfPlanSeqs)
     const int* n_items;
     unsigned int* ticket;
+    int target;                 // items aimed at (self-planning)
     int* status;
 };
+
+// Batches of up to kSelfPlanSeqs sequences need no plan kernel, no ticket and no scratch clear: every CTA derives the chunk
+// length and its items (item i -> CTA i mod grid; the items are equally long) from cu_seqlens itself, and so does the merge.
+constexpr int kSelfPlanSeqs = 32;
+__device__ __forceinline__ int dec_blocks(const int32_t* cu, int s) { return (cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN; }
+__device__ __forceinline__ int self_plan_chunk(const int32_t* cu, int S, int Hkv, int target) {
+    long long all = 0;
+    for (int s = 0; s < S; ++s) all += dec_blocks(cu, s);
+    all *= Hkv;
+    const long long chunk = (all + target - 1) / target;
+    return (int)(chunk < 1 ? 1 : chunk);
+}
+__device__ __forceinline__ int self_plan_count(const int32_t* cu, int S, int Hkv, int chunk) {
+    int k = 0;
+    for (int s = 0; s < S; ++s) k += ((dec_blocks(cu, s) + chunk - 1) / chunk) * Hkv;
+    return k;
+}
+__device__ __forceinline__ DecItem self_plan_item(const int32_t* cu, int S, int Hkv, int chunk, int item) {
+    DecItem it = {0, 0, 0, 0};
+    for (int s = 0; s < S; ++s) {
+        const int nb = dec_blocks(cu, s), per = (nb + chunk - 1) / chunk;
+        if (item < per * Hkv) {
+            const int h = item / per, i = item - h * per;
+            it.s = s; it.kvh = h; it.b0 = i * chunk; it.b1 = min((i + 1) * chunk, nb);
+            return it;
+        }
+        item -= per * Hkv;
+    }
+    return it;
+}
+__device__ __forceinline__ int2 self_plan_segment(const int32_t* cu, int S, int Hkv, int chunk, int s_want, int kvh) {
+    int first = 0;
+    for (int s = 0; s < s_want; ++s) first += ((dec_blocks(cu, s) + chunk - 1) / chunk) * Hkv;
+    const int per = (dec_blocks(cu, s_want) + chunk - 1) / chunk;
+    return make_int2(first + kvh * per, per);
+}
 
 // One CTA: per sequence the number of key blocks, a common chunk length (blocks per item) so that about
 // `target` items exist, then the items of every (sequence, KV head) written next to each other.
@@ -127,16 +164,23 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const uint32_t tS = tmem, tP = tmem, tO = tmem + 128;
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, kDecBN, false, false);
     constexpr uint32_t idesc_o = idesc_bf16_f32(128, D, false, true);
-    const int n_items = *p.n_items;
+    const bool self_plan = (p.plan == nullptr);
+    const int chunk = self_plan ? self_plan_chunk(p.cu, p.S, p.Hkv, p.target) : 0;
+    const int n_items = self_plan ? self_plan_count(p.cu, p.S, p.Hkv, chunk) : *p.n_items;
     uint32_t blk0 = 0, items_done = 0;       // barrier phases run on across the items of this CTA
 
     for (;;) {
-        if (tid == 0) *item_gen = (int)atomicAdd(p.ticket, 1u);
-        __syncthreads();
-        const int item = *item_gen;
+        int item;
+        if (self_plan) {
+            item = (int)blockIdx.x + (int)items_done * (int)gridDim.x;
+        } else {
+            if (tid == 0) *item_gen = (int)atomicAdd(p.ticket, 1u);
+            __syncthreads();
+            item = *item_gen;
+        }
         if (item >= n_items || *abort_gen) break;
         tc_fence_after();
-        const DecItem it = p.plan[item];
+        const DecItem it = self_plan ? self_plan_item(p.cu, p.S, p.Hkv, chunk, item) : p.plan[item];
         const int seq_a = p.cu[it.s], len = p.cu[it.s + 1] - seq_a;
         const int nblk = it.b1 - it.b0;
         const int last_blk = (len + kDecBN - 1) / kDecBN - 1;       // the block of the sequence with a ragged end
@@ -196,34 +240,44 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 if (!ok) { *abort_gen = 1; atomicExch(p.status, DASH_ERR_TIMEOUT); }
             }
         } else {
-            // ---- softmax warp: lane <-> row of the tile = query head kvh * G + lane (lanes >= G compute on zeros) ----
-            float m = -INFINITY, l = 0.f;
+            // ---- softmax warp.  Only rows 0..G-1 of the 128-row tile exist, so the scores are fetched in the 16-row shape
+            // (tcgen05.ld.16x256b): thread t holds, of row t / 4, the keys 8u + 2 (t % 4) + {0, 1} of every group u of 8 keys
+            // (and the same of row t / 4 + 8, which is not a real head and is ignored).  Four threads share a row: 32 exponentials
+            // per thread and block instead of 128.  P goes back in the 16x128b shape, whose 32-bit column 4u + (t % 4) is exactly
+            // the pair of keys the thread holds. ----
+            const int sub = lane & 3, hrow = lane >> 2;         // position within the row's four threads, row (query head of the group)
+            float m = -INFINITY, l = 0.f;                       // m: common to the row's threads, l: this thread's share
             bool ok = true;
             for (int j = 0; j < nblk; ++j) {
                 const uint32_t ph = (blk0 + j) & 1;
                 ok = mbar_wait(bar_s, ph, kDecWaitCycles);
                 if (!ok || *abort_gen) { ok = false; break; }
                 tc_fence_after();
-                uint32_t sreg[128];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, &sreg[c * 32]);
+                uint32_t raw[64];
+                tmem_ld16x256_x8(tS, &raw[0]);
+                tmem_ld16x256_x8(tS + 64, &raw[32]);
                 tmem_wait_ld();
+                float sc[32];                                   // sc[2u + e] = score of key 8u + 2 sub + e
+#pragma unroll
+                for (int u = 0; u < 16; ++u) { sc[2 * u] = __uint_as_float(raw[4 * u]); sc[2 * u + 1] = __uint_as_float(raw[4 * u + 1]); }
                 const bool ragged = (it.b0 + j == last_blk);
                 const int valid = len - (it.b0 + j) * kDecBN;               // keys of this block that exist (>= 1)
                 if (ragged) {
 #pragma unroll
-                    for (int c = 0; c < 128; ++c)
-                        if (c >= valid) sreg[c] = 0xff800000u;             // -inf: past the end of the sequence's cache
+                    for (int u = 0; u < 16; ++u) {
+                        if (8 * u + 2 * sub >= valid) sc[2 * u] = -INFINITY;         // past the end of the sequence's cache
+                        if (8 * u + 2 * sub + 1 >= valid) sc[2 * u + 1] = -INFINITY;
+                    }
                 }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < 128; c += 8) {
-                    mx0 = fmax3(mx0, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
-                    mx1 = fmax3(mx1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
-                    mx2 = fmax3(mx2, __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
-                    mx3 = fmax3(mx3, __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
+                for (int c = 0; c < 32; c += 4) {
+                    mx0 = fmax3(mx0, sc[c], sc[c + 1]);
+                    mx1 = fmax3(mx1, sc[c + 2], sc[c + 3]);
                 }
-                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                float mx = fmaxf(mx0, mx1);
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
                 // the reference max only moves when the block max exceeds it by more than 2^8 (then O is rescaled)
                 const bool grow = (mx - m) * p.scale_log2 > 8.0f;
                 const float m_new = grow ? mx : m;
@@ -233,15 +287,17 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     ok = mbar_wait(bar_o, (blk0 + j - 1) & 1, kDecWaitCycles);
                     if (!ok) break;
                     tc_fence_after();
+                    const float a_row = __shfl_sync(0xffffffffu, alpha, (lane * 4) & 31);   // lane r < 8 rescales row r of O
 #pragma unroll 1
                     for (int c = 0; c < D / 8; ++c) {
                         uint32_t o[8];
                         tmem_ld8(tO + c * 8, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * (lane < 8 ? a_row : 1.0f));
                         tmem_st8(tO + c * 8, o);
                     }
+                    tmem_wait_st();
                 }
                 if (ragged) {
                     // cached rows past the end of the sequence may hold anything: zero them (0 * garbage must not make a NaN)
@@ -259,30 +315,35 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     }
                     fence_proxy_async_smem();
                 }
-                float2 sumA = make_float2(0.f, 0.f), sumB = make_float2(0.f, 0.f);
+                float2 sum2 = make_float2(0.f, 0.f);
                 const float2 sl2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-msl, -msl);
+                uint32_t pk[32];                                // pk[2u] = P of (row, keys 8u + 2 sub + {0,1}); pk[2u + 1] = row + 8: nothing
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
 #pragma unroll
-                    for (int c = half * 64; c < half * 64 + 64; c += 4) {
-                        const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), sl2, nm2);
-                        const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), sl2, nm2);
-                        float2 pa, pb;
-                        pa.x = ex2(xa.x); pa.y = ex2(xa.y); pb.x = ex2(xb.x); pb.y = ex2(xb.y);
-                        sumA = __fadd2_rn(sumA, pa);
-                        sumB = __fadd2_rn(sumB, pb);
-                        sreg[c >> 1] = pack_bf16(pa.x, pa.y);
-                        sreg[(c >> 1) + 1] = pack_bf16(pb.x, pb.y);
+                    for (int u = half * 8; u < half * 8 + 8; ++u) {
+                        const float2 x = __ffma2_rn(make_float2(sc[2 * u], sc[2 * u + 1]), sl2, nm2);
+                        float2 pe;
+                        pe.x = ex2(x.x); pe.y = ex2(x.y);
+                        sum2 = __fadd2_rn(sum2, pe);
+                        pk[2 * u] = pack_bf16(pe.x, pe.y);
+                        pk[2 * u + 1] = 0u;
                     }
-                    tmem_st32(tP + half * 32, &sreg[half * 32]);
+                    // the first 64 keys of P go out (and their PV steps start) while the rest is still being formed
+                    tmem_st16x128_x8(tP + half * 32, &pk[half * 16]);
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(half == 0 ? bar_p0 : bar_p1);
                 }
-                l = l * alpha + ((sumA.x + sumA.y) + (sumB.x + sumB.y));
+                l = l * alpha + (sum2.x + sum2.y);
                 m = m_new;
             }
             if (ok) ok = mbar_wait(bar_o, (blk0 + nblk - 1) & 1, kDecWaitCycles);
+            // row sum: the four threads' shares; then lane r < G writes row r (its m and l sit in thread 4 r)
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const float m_row = __shfl_sync(0xffffffffu, m, (lane * 4) & 31), l_row = __shfl_sync(0xffffffffu, l, (lane * 4) & 31);
+            (void)hrow;
             if (ok && !*abort_gen) {
                 tc_fence_after();
                 float* dst = p.partial + ((size_t)item * kDecRows + lane) * (D + 2);
@@ -297,7 +358,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                             *reinterpret_cast<float2*>(dst + c * 32 + e) = make_float2(__uint_as_float(o[e]), __uint_as_float(o[e + 1]));
                     }
                 }
-                if (lane < p.G) { dst[D] = m; dst[D + 1] = l; }
+                if (lane < p.G) { dst[D] = m_row; dst[D + 1] = l_row; }
             } else if (!ok && lane == 0) {
                 *abort_gen = 1;
                 atomicExch(p.status, DASH_ERR_TIMEOUT);
@@ -317,33 +378,36 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 }
 
 // One CTA per (sequence, query head): combine the partial results of the key splits.  The weights of the splits are formed
-// in parallel over the splits, then every thread sums its column over them (independent loads).
-constexpr int kMergeMaxSplits = 1024;
+// in parallel over the splits; the sums over the splits run in kMergeGroups thread groups (each takes every kMergeGroups-th split,
+// independent loads, unrolled) that meet in shared memory.
+constexpr int kMergeMaxSplits = 1024, kMergeGroups = 4, kMergeThreads = 128 * kMergeGroups;
 template <bool OUT_F32>
-__global__ void __launch_bounds__(128)
-decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ seg, int Hq, int G, int D,
-                    float scale_log2, float scale, void* __restrict__ out, int64_t ldo, float* __restrict__ lse) {
+__global__ void __launch_bounds__(kMergeThreads)
+decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ seg, const int32_t* __restrict__ cu, int S, int target,
+                    int Hq, int G, int D, float scale_log2, float scale, void* __restrict__ out, int64_t ldo, float* __restrict__ lse) {
     __shared__ float s_w[kMergeMaxSplits];
-    __shared__ float s_red[4];
+    __shared__ float s_red[kMergeThreads / 32];
+    __shared__ float s_acc[kMergeGroups][128];
     __shared__ float s_m, s_l;
     const int s = blockIdx.x / Hq, h = blockIdx.x % Hq;
     const int kvh = h / G, row = h % G, Hkv = Hq / G;
-    const int2 sg = seg[s * Hkv + kvh];
+    const int2 sg = seg ? seg[s * Hkv + kvh] : self_plan_segment(cu, S, Hkv, self_plan_chunk(cu, S, Hkv, target), s, kvh);
     const int cnt = sg.y < kMergeMaxSplits ? sg.y : kMergeMaxSplits;
     const size_t stride = (size_t)kDecRows * (D + 2);
     const float* base = partial + ((size_t)sg.x * kDecRows + row) * (D + 2);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    constexpr int NW = kMergeThreads / 32;
     float mx = -INFINITY;
-    for (int i = threadIdx.x; i < cnt; i += blockDim.x) mx = fmaxf(mx, base[i * stride + D]);
+    for (int i = threadIdx.x; i < cnt; i += kMergeThreads) mx = fmaxf(mx, base[i * stride + D]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (lane == 0) s_red[w] = mx;
     __syncthreads();
-    if (threadIdx.x == 0) s_m = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+    if (threadIdx.x == 0) { float v = s_red[0]; for (int i = 1; i < NW; ++i) v = fmaxf(v, s_red[i]); s_m = v; }
     __syncthreads();
     const float mall = s_m;
     float ls = 0.f;
-    for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+    for (int i = threadIdx.x; i < cnt; i += kMergeThreads) {
         const float wi = exp2f((base[i * stride + D] - mall) * scale_log2);
         s_w[i] = wi;
         ls += wi * base[i * stride + D + 1];
@@ -353,14 +417,22 @@ decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ 
     __syncthreads();
     if (lane == 0) s_red[w] = ls;
     __syncthreads();
-    if (threadIdx.x == 0) s_l = (s_red[0] + s_red[1]) + (s_red[2] + s_red[3]);
+    if (threadIdx.x == 0) { float v = 0.f; for (int i = 0; i < NW; ++i) v += s_red[i]; s_l = v; }
     __syncthreads();
     const float lall = s_l;
-    for (int c = threadIdx.x; c < D; c += blockDim.x) {
-        float acc = 0.f;
+    const int grp = threadIdx.x >> 7, c = threadIdx.x & 127;       // D <= 128: one column per thread of a group
+    float acc = 0.f;
+    if (c < D) {
 #pragma unroll 8
-        for (int i = 0; i < cnt; ++i) acc += s_w[i] * base[i * stride + c];
-        const float v = cnt > 0 ? acc / lall : 0.f;
+        for (int i = grp; i < cnt; i += kMergeGroups) acc += s_w[i] * base[i * stride + c];
+    }
+    s_acc[grp][c] = acc;
+    __syncthreads();
+    if (grp == 0 && c < D) {
+        float v = 0.f;
+#pragma unroll
+        for (int gI = 0; gI < kMergeGroups; ++gI) v += s_acc[gI][c];
+        v = cnt > 0 ? v / lall : 0.f;
         if (OUT_F32) reinterpret_cast<float*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = v;
         else reinterpret_cast<__nv_bfloat16*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = __float2bfloat16(v);
     }
@@ -433,8 +505,12 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
     int2* seg = (int2*)(w + 256 + align_up((size_t)max_items * sizeof(DecItem), 256));
     int* seq_first = (int*)((char*)seg + align_up((size_t)S * Hkv * sizeof(int2), 256));
     float* partial = (float*)((char*)seq_first + align_up((size_t)S * sizeof(int), 256));
-    decode_plan_kernel<<<1, 256, 0, st>>>(cu_seqlens, S, Hkv, 4 * sm_count(), plan, seg, (int*)(w + 4), (unsigned int*)w, max_items, seq_first);
-    DASH_CUDA_TRY(cudaGetLastError());
+    const bool self_plan = S <= kSelfPlanSeqs;
+    const int target = 4 * sm_count();
+    if (!self_plan) {
+        decode_plan_kernel<<<1, 256, 0, st>>>(cu_seqlens, S, Hkv, target, plan, seg, (int*)(w + 4), (unsigned int*)w, max_items, seq_first);
+        DASH_CUDA_TRY(cudaGetLastError());
+    }
     const float scale_log2 = scale * 1.4426950408889634f;
     if (n > 0) {
         CUtensorMap mq, mk, mv;
@@ -446,7 +522,8 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
         DecParams p;
         p.cu = cu_seqlens; p.S = S; p.Hq = Hq; p.Hkv = Hkv; p.G = G;
         p.scale = scale; p.scale_log2 = scale_log2;
-        p.partial = partial; p.plan = plan; p.n_items = (const int*)(w + 4); p.ticket = (unsigned int*)w;
+        p.partial = partial; p.plan = self_plan ? nullptr : plan; p.n_items = (const int*)(w + 4); p.ticket = (unsigned int*)w;
+        p.target = target;
         p.status = status_word_ptr();
         if (!p.status) return DASH_ERR_CUDA;
         int grid = 2 * sm_count();
@@ -454,7 +531,8 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
         rc = D == 128 ? launch_decode<128>(mq, mk, mv, p, box_heads, grid, st) : launch_decode<64>(mq, mk, mv, p, box_heads, grid, st);
         if (rc != DASH_OK) return rc;
     }
-    decode_merge_kernel<false><<<S * Hq, 128, 0, st>>>(partial, seg, Hq, G, D, scale_log2, scale, out, ldo, lse);
+    decode_merge_kernel<false><<<S * Hq, kMergeThreads, 0, st>>>(partial, self_plan ? nullptr : seg, cu_seqlens, S, target, Hq, G, D, scale_log2, scale, out,
+                                                                ldo, lse);
     DASH_CUDA_TRY(cudaGetLastError());
     return DASH_OK;
 }

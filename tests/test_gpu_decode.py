@@ -49,6 +49,15 @@ def test_decode_qwen_heads_long_cache_split_over_many_ctas():
     _decode_case([100000], 28, 4, 128, 3)
 
 
+def test_decode_large_batch_takes_the_planned_path():
+    # more sequences than the CTAs plan for themselves: items come from the plan kernel, by ticket
+    g = torch.Generator().manual_seed(6)
+    lengths = torch.randint(0, 700, (45,), generator=g).tolist()
+    lengths[3] = 0
+    lengths[10] = 9000
+    _decode_case(lengths, 14, 2, 128, 6, pad=7)
+
+
 def test_decode_head_dim_64_no_grouping_and_wide_grouping():
     _decode_case([777, 2000], 4, 4, 64, 4)
     _decode_case([1500], 8, 1, 64, 5, pad=3)
