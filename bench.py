@@ -19,6 +19,9 @@ its own batch (weak scaling, no data-path collective).
 feed-forward, selection at block 11, compression ratio 0.667): a step = the whole prefill, and the
 dense prefill is timed beside it for the measured speedup next to the Appendix-A FLOPs model.
 
+`--workload decode --seq T`: the decoding stage over the KV caches that prefill leaves (attention of one new token over all 28
+caches, dense and shortened).
+
 Prints one JSON line (rank 0).  `--impl reference` times the CPU oracle, as it stands, on
 the host cores on a bounded sample of the cfg2 workload.
 """
@@ -545,6 +548,71 @@ def setup_stack(args, dash, dev, rank):
     }
 
 
+def setup_decode(args, dash, dev, rank):
+    """Decoding stage over the KV caches a halted prefill leaves behind (28 blocks, selection at block 11, compression ratio
+    0.667 as in the paper's efficiency setting): blocks 1..11 cache all T prompt tokens, blocks 12..28 only the tokens that
+    stayed.  A step = the attention of one new token over all 28 caches; the dense caches are timed beside it."""
+    T, Lr, l_s, rho = args.seq, 28, 11, 0.667
+    sh, S = wl.QWEN, 1
+    K = dash.dash_keep_count(T, rho, 64, 32, 1)
+    g = torch.Generator(device=dev).manual_seed(rank_seed(6, rank))
+    # every block has its own cache, as a real KV cache has (28 x 268 MB at 131072 tokens): the decoding step streams them from HBM
+    def cache(n_l):
+        return (torch.randn(n_l, sh.Hkv, sh.D, device=dev, generator=g).to(sh.dtype), torch.randn(n_l, sh.Hkv, sh.D, device=dev, generator=g).to(sh.dtype))
+    dense = [cache(T) for _ in range(Lr)]
+    halted = dense[:l_s] + [cache(K) for _ in range(Lr - l_s)]
+    Kc, Vc = dense[0]
+    q_host = _pin(torch.randn(S, sh.Hq, sh.D).to(sh.dtype))
+    q = torch.empty_like(q_host, device=dev)
+    out = torch.empty(S, sh.Hq, sh.D, dtype=sh.dtype, device=dev)
+    out_h = _pin(torch.empty(S, sh.Hq, sh.D, dtype=sh.dtype))
+    cu_full = torch.tensor([0, T], dtype=torch.int32, device=dev)
+    cu_kept = torch.tensor([0, K], dtype=torch.int32, device=dev)
+    ws = dash.workspace(dash.dash_workspace_bytes(dash.WS_DECODE, T, S, sh.Hq, sh.Hkv, sh.D), dev)
+
+    def attn_over(halting):
+        for l in range(Lr):
+            kc, vc = (halted if halting else dense)[l]
+            dash.dash_decode_attention(q, kc, vc, cu_kept if kc.shape[0] == K else cu_full, out=out, ws=ws)
+
+    def h2d():
+        q.copy_(q_host, non_blocking=True)
+
+    def d2h():
+        out_h.copy_(out, non_blocking=True)
+
+    h2d()
+    t_full = timer_simple(lambda: attn_over(False), 5)
+    t_halt = timer_simple(lambda: attn_over(True), 5)
+    row_b = 2 * sh.Hkv * sh.D * 2                              # K and V bytes per cached token and block
+    kv_full, kv_halt = Lr * T * row_b, (l_s * T + (Lr - l_s) * K) * row_b
+    U = torch.randn(T, sh.d, device=dev).to(sh.dtype); Hh = torch.randn(T, sh.d, device=dev).to(sh.dtype); Ht = torch.empty_like(Hh)
+    r, mask = torch.zeros(T, device=dev), torch.zeros(T, dtype=torch.uint8, device=dev)
+    mask2 = wl.random_mask(T, 0.333, seed=7).to(dev)
+    k2 = int(mask2.sum().item())
+    Hn = torch.empty_like(Hh)
+    pos = torch.arange(T, dtype=torch.int32, device=dev)
+    cws = dash.workspace(dash.dash_workspace_bytes(dash.WS_COMPACT, T, S), dev)
+    oo = {"pos_out": torch.empty_like(pos), "tok_out": torch.empty_like(pos), "cu_out": torch.empty(2, dtype=torch.int32, device=dev),
+          "n_out": torch.empty(1, dtype=torch.int32, device=dev)}
+    extra = {"blocks": Lr, "start_block": l_s, "kept_length": K, "kv_cache_bytes_dense": kv_full, "kv_cache_bytes_halted": kv_halt,
+             "kv_cache_ratio": kv_halt / kv_full, "dense_decode_attention_ms": t_full, "halted_decode_attention_ms": t_halt,
+             "speedup_measured": t_full / t_halt,
+             "value_counts": "new tokens per second of the attention part of one decoding step over all 28 caches (batch 1)"}
+    return {
+        "workload": f"decoding stage after a halted prefill of {T} tokens: attention of one new token over the KV caches of {Lr} "
+                    f"Qwen2.5-7B-shaped blocks ({l_s} with {T} cached tokens, {Lr - l_s} with {K}), bf16, batch 1",
+        "dtype": "bf16", "step": (lambda: attn_over(True)), "h2d": h2d, "d2h": d2h, "tokens": 1, "launches": 2 * Lr,
+        "launch_note": f"{Lr} x (decode kernel, merge kernel)",
+        "h2d_bytes": _bytes(q_host), "d2h_bytes": _bytes(out_h), "extra": extra,
+        "attn": (lambda: dash.dash_decode_attention(q, Kc, Vc, cu_full, out=out, ws=ws)), "attn_flops": 4.0 * sh.Hq * sh.D * T,
+        "attn_bytes": float(T * row_b), "attn_name": f"decode_kernel<{sh.D}> + merge over {T} cached tokens (HBM-bound: K and V read once)",
+        "norm": (lambda: dash.dash_delta_norm(U, Hh, r_out=r, Hres_out=Ht, tau=0.0, cu_seqlens=cu_full, mask_out=mask)), "norm_bytes": T * (3 * sh.d * 2 + 5),
+        "compact": (lambda: dash.dash_compact(mask2, cu_full, rows=[Ht], rows_out=[Hn], pos_in=pos, tok_in=pos, want_idx=False, ws=cws, outputs=oo)),
+        "compact_bytes": k2 * (2 * sh.d * 2 + 16) + T * 9, "compact_rows": k2, "row_bytes": sh.d * 2,
+    }
+
+
 def timer_simple(fn, reps):
     """Mean device time (ms) of fn over reps runs, after one untimed run."""
     fn(); torch.cuda.synchronize()
@@ -586,7 +654,7 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    setup = {"cfg1": setup_block_step, "cfg2": setup_block_step, "cfg3": setup_cascade, "cfg4": setup_sparse, "cfg5": setup_sparse, "stack": setup_stack}[args.workload]
+    setup = {"cfg1": setup_block_step, "cfg2": setup_block_step, "cfg3": setup_cascade, "cfg4": setup_sparse, "cfg5": setup_sparse, "stack": setup_stack, "decode": setup_decode}[args.workload]
     W = setup(args, dash, dev, rank)
     step = W["step"]
     for _ in range(max(args.warmup, 3)):
@@ -651,9 +719,13 @@ def run_ours(args):
         "e2e": e2e_entry(tokens, world, t_e2e, t_pipe, W["h2d_bytes"], W["d2h_bytes"]),
         "gpu_launches": W["launches"] * args.steps, "gpu_launches_note": W["launch_note"],
         "clocks": clocks,
-        "roofline": {"kernel": W["attn_name"], "bound": "tensor", "achieved": ach,
-                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"], "peak_source": peaks["source"],
-                     "frac_of_nominal_2250": ach / 2250.0, "ms_per_launch": t_attn, "flops_per_launch": fl, "traffic": ATTN_TRAFFIC.get(args.workload)},
+        "roofline": ({"kernel": W["attn_name"], "bound": "tensor", "achieved": ach,
+                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"], "peak_source": peaks["source"],
+                      "frac_of_nominal_2250": ach / 2250.0, "ms_per_launch": t_attn, "flops_per_launch": fl, "traffic": ATTN_TRAFFIC.get(args.workload)}
+                     if "attn_bytes" not in W else
+                     {"kernel": W["attn_name"], "bound": "hbm", "achieved": W["attn_bytes"] / (t_attn * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                      "unit": "GB/s", "frac": W["attn_bytes"] / (t_attn * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                      "ms_per_launch": t_attn, "bytes_per_launch": W["attn_bytes"], "traffic": None}),
         "hbm_kernels": {
             "delta_norm_fused": hbm(ms_norm, W["norm_bytes"]), "compact": hbm(ms_comp, W["compact_bytes"]),
             "contiguous_copy_of_the_compacted_bytes": hbm(ms_copy, 2 * nrow * W["row_bytes"]),
@@ -747,7 +819,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "stack"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "stack", "decode"],
                     help="cfg2 (default) is the configuration the headline metric is quoted on; the others are the remaining benchmark configurations")
     ap.add_argument("--seq", type=int, default=None, help="tokens per sequence (cfg1: 1024, cfg2: 8192, cfg3: 32768)")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
@@ -757,6 +829,8 @@ def main():
         args.seq = {"cfg1": 1024, "cfg2": 8192, "cfg3": 32768}.get(args.workload, 8192)
     if args.workload == "stack":
         args.steps = min(args.steps, 5)                 # a step is a whole 28-block prefill
+    if args.workload == "decode":
+        args.steps = min(args.steps, 50)
     if args.impl == "reference":
         run_reference(args)
     else:
