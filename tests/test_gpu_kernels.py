@@ -260,3 +260,55 @@ def test_attention_closed_forms_on_device():
     O = dash.dash_varlen_attention(torch.zeros_like(Q), K, V, cu, n)
     pm = torch.cumsum(V.float()[:, 0], 0) / torch.arange(1, n + 1, device=DEV)[:, None]
     assert torch.allclose(O.float()[:, 1], pm, atol=2e-2)
+
+
+# ------------------------------------------------------------------ randomized sweeps (seeded)
+def test_select_compact_scatter_random_shapes_match_oracle():
+    """Thirty seeded draws of batch structure, keep ratio, rule and protected tokens: select, compaction and scatter against the oracle."""
+    g = torch.Generator().manual_seed(2024)
+    for trial in range(30):
+        S = int(torch.randint(1, 7, (1,), generator=g))
+        lengths = [int(x) for x in torch.randint(0, [40, 400, 5000, 40000][trial % 4], (S,), generator=g)]
+        if sum(lengths) == 0:
+            lengths[0] = 17
+        cu = wl.cu_from_lengths(lengths)
+        n = int(cu[-1])
+        r = torch.rand(n, generator=g)
+        kf, kl = int(torch.randint(0, 5, (1,), generator=g)), int(torch.randint(0, 5, (1,), generator=g))
+        mode = [dash.SEL_THRESHOLD, dash.SEL_KEEP_COUNT, dash.SEL_THRESHOLD_HALT_HIGH, dash.SEL_KEEP_COUNT_HALT_HIGH][trial % 4]
+        keep = float(torch.rand(1, generator=g))
+        K = [min(L, int(keep * L) + int(torch.randint(0, 3, (1,), generator=g))) for L in lengths]
+        kc = torch.tensor(K, dtype=torch.int32, device=DEV)
+        m = dash.dash_select(r.to(DEV), cu.to(DEV), mode, tau=keep, keep_counts=kc, keep_first=kf, keep_last=kl)
+        ref = oc.select(r.numpy(), cu, oc.THRESHOLD if mode in (dash.SEL_THRESHOLD, dash.SEL_THRESHOLD_HALT_HIGH) else oc.KEEP_COUNT,
+                        tau=keep, keep_counts=K, keep_first=kf, keep_last=kl, halt_high=mode >= 2)
+        assert np.array_equal(m.cpu().numpy(), ref), (trial, lengths, mode)
+        d = [8, 24, 256, 520][trial % 4]
+        X = torch.randn(n, d, generator=g).to(torch.bfloat16 if trial % 2 else torch.float32)
+        pos = wl.positions(cu)
+        tok = torch.randperm(n, generator=g).to(torch.int32)
+        c = dash.dash_compact(m, cu.to(DEV), rows=[X.to(DEV)], pos_in=pos.to(DEV), tok_in=tok.to(DEV))
+        o = oc.compact(ref, cu, rows=[X], pos_in=pos, tok_in=tok)
+        k = int(c["n_out"].item())
+        assert k == o["n_out"] and np.array_equal(c["cu_out"].cpu().numpy(), o["cu_out"]), (trial, lengths)
+        assert np.array_equal(c["idx"][:k].cpu().numpy(), o["idx"])
+        assert torch.equal(c["rows"][0][:k].cpu(), o["rows"][0])
+        assert np.array_equal(c["pos_out"][:k].cpu().numpy(), o["pos_out"]) and np.array_equal(c["tok_out"][:k].cpu().numpy(), o["tok_out"])
+        full = torch.zeros(n, d, dtype=X.dtype, device=DEV)
+        dash.dash_scatter(X.to(DEV), full, tok_index=tok.to(DEV), sel=m, which=trial % 3)
+        want = oc.scatter(X, tok, ref, trial % 3, torch.zeros(n, d, dtype=X.dtype))
+        assert torch.equal(full.cpu(), want), (trial, "scatter")
+
+
+def test_attention_random_packed_batches_match_oracle_on_sampled_rows():
+    g = torch.Generator().manual_seed(77)
+    for trial in range(6):
+        S = int(torch.randint(1, 6, (1,), generator=g))
+        lengths = [int(x) for x in torch.randint(0, 900, (S,), generator=g)]
+        if sum(lengths) == 0:
+            lengths[0] = 130
+        Hkv = [1, 2, 4][trial % 3]
+        Hq = Hkv * [1, 3, 7][trial % 3]
+        D = 128 if trial % 2 else 64
+        rows = wl.sample_rows(wl.cu_from_lengths(lengths), 60, seed=trial)
+        _attention_case(lengths, Hq, Hkv, D, torch.bfloat16, 100 + trial, rows=rows.numpy(), pad=trial)
