@@ -215,7 +215,8 @@ def setup_block_step(args, dash, dev, rank):
     pos, tok = torch.empty(T, dtype=torch.int32, device=dev), torch.empty(T, dtype=torch.int32, device=dev)
     cu = torch.empty(S + 1, dtype=torch.int32, device=dev)
     x_full = torch.zeros(T, sh.d, dtype=sh.dtype, device=dev)
-    dev_out = (x_full, B.H_next, B.r, B.mask, B.tok_next, B.cu_next)
+    # results read back: H_next is not among them -- its rows are rows of x_full (H_next[k] = x_full[tok_next[k]]), so the host has them
+    dev_out = (x_full, B.r, B.mask, B.tok_next, B.cu_next)
     host_out = [_pin(torch.empty_like(t, device="cpu")) for t in dev_out]
 
     def h2d():
@@ -237,7 +238,7 @@ def setup_block_step(args, dash, dev, rank):
         ins = [(H, pos, tok, cu), tuple(torch.empty_like(t) for t in (H, pos, tok, cu))]
         xs = [x_full, torch.zeros_like(x_full)]
         bs = [B, B2]
-        outs_d = [dev_out, (xs[1], B2.H_next, B2.r, B2.mask, B2.tok_next, B2.cu_next)]
+        outs_d = [dev_out, (xs[1], B2.r, B2.mask, B2.tok_next, B2.cu_next)]
         outs_h = [host_out, [_pin(torch.empty_like(t, device="cpu")) for t in outs_d[1]]]
         s_c, s_in, s_out = torch.cuda.current_stream(), torch.cuda.Stream(), torch.cuda.Stream()
         ev_in = [torch.cuda.Event() for _ in range(2)]
