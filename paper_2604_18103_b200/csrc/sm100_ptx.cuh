@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the attention and GEMM
-// kernels use: mbarrier, TMA tiled loads (never multicast), tcgen05 MMA with
+// kernels use: mbarrier, TMA tiled loads (each CTA fetches its own tiles), tcgen05 MMA with
 // TMEM accumulators, TMEM loads/stores, and the shared-memory / instruction
 // descriptors of tcgen05.mma.
 #pragma once
