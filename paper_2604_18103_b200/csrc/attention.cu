@@ -49,19 +49,6 @@ int make_map_rows_heads(CUtensorMap* map, const void* base, int64_t rows, int he
     return r == CUDA_SUCCESS ? DASH_OK : DASH_ERR_CUDA;
 }
 
-int make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return DASH_ERR_CUDA;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? DASH_OK : DASH_ERR_CUDA;
-}
-
 constexpr int kBM = 128;                 // query rows per CTA
 constexpr int kBN = 128;                 // keys per block
 constexpr int kAttnThreads = 160;

@@ -14,7 +14,6 @@
 
 namespace dash {
 
-constexpr int kWarp = 32;
 // polls before a device-side wait gives up and records DASH_ERR_TIMEOUT
 constexpr uint32_t kSpinLimit = 1u << 22;
 
@@ -37,10 +36,6 @@ __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
 }
 __device__ __forceinline__ void st_v4(void* p, uint4 v) {
     asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-// streaming store: written once, not re-read by this kernel
-__device__ __forceinline__ void st_cs_v4(void* p, uint4 v) {
-    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

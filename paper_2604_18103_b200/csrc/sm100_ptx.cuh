@@ -1,5 +1,4 @@
-// Thin inline-PTX wrappers for the sm_100a features the attention and GEMM
-// kernels use: mbarrier, TMA tiled loads (each CTA fetches its own tiles), tcgen05 MMA with
+// Thin inline-PTX wrappers for the sm_100a features the attention kernels use: mbarrier, TMA tiled loads (each CTA fetches its own tiles), tcgen05 MMA with
 // TMEM accumulators, TMEM loads/stores, and the shared-memory / instruction
 // descriptors of tcgen05.mma.
 #pragma once
@@ -57,19 +56,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const CUtensorMap
         ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src_smem, int c0, int c1) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src_smem), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // ---- TMEM allocation (one full warp executes these) -------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
@@ -223,7 +209,5 @@ EncodeTiledFn encode_tiled_fn();
 
 // bf16 tensor [rows, heads, D] with row stride ld (elements): box = 64 x 1 x box_rows, 128-byte swizzle
 int make_map_rows_heads(CUtensorMap* map, const void* base, int64_t rows, int heads, int D, int64_t ld, int box_rows);
-// bf16 matrix [rows, cols] with row stride ld (elements): box = 64 x box_rows, 128-byte swizzle
-int make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows);
 
 }  // namespace dash
