@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdash.so")
-SOURCES = ["api.cu", "hbm_kernels.cu", "attention.cu", "decode_attention.cu", "layer_step.cu"]
+SOURCES = ["api.cu", "hbm_kernels.cu", "attention.cu", "decode_attention.cu", "gemm.cu", "layer_step.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC] + os.environ.get("DASH_NVCC_EXTRA", "").split()

@@ -1,0 +1,33 @@
+// Internal interface of the projection GEMMs (gemm.cu).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dash.h"
+
+namespace dash {
+
+enum GemmEpilogueKind { GEMM_PLAIN = 0, GEMM_ROPE = 1, GEMM_RESID = 2, GEMM_SWIGLU = 3 };
+
+struct GemmEpilogue {
+    // ROPE: heads of D columns; columns below n_rot_cols (a multiple of 256) belong to Q and K heads and are rotated with
+    // rope_table [n, D/2] = (cos, sin) of every row
+    int D = 0, n_rot_cols = 0;
+    const float2* rope_table = nullptr;
+    // RESID: x_full[tok_index[row]] (tok_index null: row) = H[row] + (A W)[row]; sums [n, N/256] = (sum u^2, sum h^2) per column tile
+    const void* H = nullptr; int64_t ldh = 0;
+    const int32_t* tok_index = nullptr;
+    void* x_full = nullptr; int64_t ldx = 0;
+    float2* sums = nullptr;
+    // SWIGLU: W = [K, 2m] (gate | up); C [n, m] = silu(A Wg) * (A Wu)
+    int m = 0;
+};
+
+// true if the own kernel takes this problem (bf16, 256-column tiles, K in steps of 64); otherwise the caller uses the library GEMM
+bool gemm_shape_ok(GemmEpilogueKind kind, int64_t n, int64_t N, int64_t K, int64_t lda, int64_t ldw, const GemmEpilogue& e);
+// C (or the epilogue's outputs) = A[n, K] W[K, N]; ld* in elements; n_dev: device true row count or null
+int gemm_bf16(GemmEpilogueKind kind, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc, int64_t n, int64_t N,
+              int64_t K, const GemmEpilogue& e, const int32_t* n_dev, cudaStream_t st);
+int launch_rope_table(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const int32_t* n_dev, cudaStream_t st);
+
+}  // namespace dash

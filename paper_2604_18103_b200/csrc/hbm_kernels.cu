@@ -439,6 +439,8 @@ __device__ __forceinline__ uint4 ld_cg_v4(const void* p) {
 struct TailArgs {
     const char* U; const char* H; int64_t ldU_b, ldH_b; int nvec; int mode; float eps;
     const uint8_t* mask_in;       // non-null: keep decisions are given (r and the mask are not formed), U is any update to add to H
+    const float2* sums; int n_sum_tiles;   // non-null: per-row partial (sum u^2, sum h^2) from the output-projection epilogue; with U null
+                                           // the rows are already in x_full and only the score, the decision and the compaction remain
     float tau; int keep_first, keep_last; const int32_t* cu_in; int S;
     const int32_t* tok_in; const int32_t* pos_in;
     char* x_full; int64_t ldx_b; char* H_next; int64_t ldn_b;
@@ -471,30 +473,37 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
         const int64_t row = t_start + local;
         int keep = 0;
         if (row < n) {
-            const char* u = a.U + row * a.ldU_b;
-            const char* h = a.H + row * a.ldH_b;
-            char* o = a.x_full + (int64_t)a.tok_in[row] * a.ldx_b;
             float su = 0.f, sh = 0.f;
-            for (int base = 0; base < a.nvec; base += 32 * CH) {
-                uint4 x[CH], y[CH];
+            if (a.U) {
+                const char* u = a.U + row * a.ldU_b;
+                const char* h = a.H + row * a.ldH_b;
+                char* o = a.x_full + (int64_t)a.tok_in[row] * a.ldx_b;
+                for (int base = 0; base < a.nvec; base += 32 * CH) {
+                    uint4 x[CH], y[CH];
 #pragma unroll
-                for (int k = 0; k < CH; ++k) {
-                    const int v = base + k * 32 + lane;
-                    if (v < a.nvec) { x[k] = ld_nc_v4(u + ((int64_t)v << 4)); y[k] = ld_nc_v4(h + ((int64_t)v << 4)); }
-                }
+                    for (int k = 0; k < CH; ++k) {
+                        const int v = base + k * 32 + lane;
+                        if (v < a.nvec) { x[k] = ld_nc_v4(u + ((int64_t)v << 4)); y[k] = ld_nc_v4(h + ((int64_t)v << 4)); }
+                    }
 #pragma unroll
-                for (int k = 0; k < CH; ++k) {
-                    const int v = base + k * 32 + lane;
-                    if (v < a.nvec) {
-                        su += sumsq_vec<BF16>(x[k]);
-                        sh += sumsq_vec<BF16>(y[k]);
-                        st_v4(o + ((int64_t)v << 4), add_vec<BF16>(x[k], y[k]));
+                    for (int k = 0; k < CH; ++k) {
+                        const int v = base + k * 32 + lane;
+                        if (v < a.nvec) {
+                            su += sumsq_vec<BF16>(x[k]);
+                            sh += sumsq_vec<BF16>(y[k]);
+                            st_v4(o + ((int64_t)v << 4), add_vec<BF16>(x[k], y[k]));
+                        }
                     }
                 }
             }
             if (a.mask_in) {
                 keep = a.mask_in[row] != 0;
             } else {
+                if (a.sums) {
+                    // the projection's column tiles, summed in a fixed order (lane i takes tiles i, i + 32, ...)
+                    su = 0.f; sh = 0.f;
+                    for (int i = lane; i < a.n_sum_tiles; i += 32) { const float2 p2 = a.sums[(int64_t)row * a.n_sum_tiles + i]; su += p2.x; sh += p2.y; }
+                }
                 su = warp_sum(su);
                 sh = warp_sum(sh);
                 const float num = sqrtf(su);
@@ -780,9 +789,40 @@ extern "C" int dash_compact_static(const uint8_t* mask, int64_t n, const int32_t
 namespace dash {
 size_t select_ws_bytes(int64_t, int) { return 256; }
 
+// r (and, with ft.mask_out set, the threshold decision) from the per-row partial sums of the output-projection epilogue
+__global__ void __launch_bounds__(256)
+sums_to_score_kernel(const float2* __restrict__ sums, int n_sum_tiles, int64_t n, int mode, float eps, float* __restrict__ r_out,
+                     FusedThreshold ft, const int32_t* __restrict__ n_dev) {
+    if (n_dev) { int64_t nd = *n_dev; if (nd < n) n = nd; }
+    for (int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; row < n; row += (int64_t)gridDim.x * blockDim.x) {
+        float su = 0.f, sh = 0.f;
+        for (int i = 0; i < n_sum_tiles; ++i) { const float2 p2 = sums[row * n_sum_tiles + i]; su += p2.x; sh += p2.y; }
+        const float num = sqrtf(su);
+        const float r = (mode == DASH_NORM_ABS) ? num : num / fmaxf(sqrtf(sh), eps);
+        r_out[row] = r;
+        if (ft.mask_out) {
+            const int s = find_seq(ft.cu, ft.S, (int)row);
+            const int local = (int)row - ft.cu[s], len = ft.cu[s + 1] - ft.cu[s];
+            const bool prot = (local < ft.keep_first) || (local >= len - ft.keep_last);
+            ft.mask_out[row] = (prot || !(r < ft.tau)) ? 1 : 0;
+        }
+    }
+}
+
+int launch_sums_to_score(const float2* sums, int n_sum_tiles, int64_t n, dash_norm_mode mode, float eps, float* r_out, const dash_threshold* fused,
+                         const int32_t* n_dev, cudaStream_t st) {
+    FusedThreshold ft = {0.f, 0, 0, nullptr, 0, nullptr};
+    if (fused) ft = {fused->tau, fused->keep_first, fused->keep_last, fused->cu_seqlens, fused->S, fused->mask_out};
+    int64_t blocks = (n + 255) / 256, cap = (int64_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    sums_to_score_kernel<<<(int)blocks, 256, 0, st>>>(sums, n_sum_tiles, n, (int)mode, eps, r_out, ft, n_dev);
+    return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+}
+
 // Fused tail of the block step (see delta_tail_kernel).  Preconditions checked by the caller: threshold rule, every row
 // scattered, 16-byte aligned rows.  ws: the compaction workspace (ticket + one state word per 32-token tile).
-int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
+int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float2* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
                       int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st) {
@@ -791,7 +831,7 @@ int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, int6
     const int tiles = (int)((n + 31) / 32) > 0 ? (int)((n + 31) / 32) : 1;
     DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)tiles * 8, st));
     TailArgs a;
-    a.mask_in = mask_in;
+    a.mask_in = mask_in; a.sums = sums; a.n_sum_tiles = n_sum_tiles;
     a.U = (const char*)U; a.H = (const char*)H; a.ldU_b = a.ldH_b = (int64_t)d * es; a.nvec = d * es / 16; a.mode = (int)mode; a.eps = eps;
     a.tau = tau; a.keep_first = keep_first; a.keep_last = keep_last; a.cu_in = cu_in; a.S = S; a.tok_in = tok_in; a.pos_in = pos_in;
     a.x_full = (char*)x_full; a.ldx_b = (int64_t)d * es; a.H_next = (char*)H_next; a.ldn_b = (int64_t)d * es;

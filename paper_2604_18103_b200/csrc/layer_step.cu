@@ -12,6 +12,7 @@
 #include <tuple>
 
 #include "common.cuh"
+#include "gemm.cuh"
 
 namespace dash {
 
@@ -165,10 +166,21 @@ static int gemm_rowmajor(dash_dtype dt, const void* A, int64_t lda, const void* 
     return rc;
 }
 
-int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
+int launch_sums_to_score(const float2* sums, int n_sum_tiles, int64_t n, dash_norm_mode mode, float eps, float* r_out, const dash_threshold* fused,
+                         const int32_t* n_dev, cudaStream_t st);
+int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float2* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
                       int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st);
+
+// C = A W: this library's GEMM when it takes the problem (bf16, 256-column tiles), the library GEMM otherwise
+static int project(bool own, dash_dtype dt, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc, int64_t n, int64_t N, int64_t K,
+                   const int32_t* n_dev, void* lt_ws, cudaStream_t st) {
+    GemmEpilogue e;
+    if (own && dt == DASH_BF16 && gemm_shape_ok(GEMM_PLAIN, n, N, K, lda, ldw, e) && aligned16(C) && (ldc % 8) == 0)
+        return gemm_bf16(GEMM_PLAIN, A, lda, W, ldw, C, ldc, n, N, K, e, n_dev, st);
+    return gemm_rowmajor(dt, A, lda, W, ldw, C, ldc, n, N, K, lt_ws, st);
+}
 
 static int rows_grid8(int64_t n) {
     int64_t blocks = (n + 7) / 8, cap = (int64_t)sm_count() * 8;
@@ -219,6 +231,7 @@ static bool cfg_ok(const dash_layer_cfg* c) {
     if (c->scatter_which != 0 && c->scatter_which != 2) return false;
     if (!(c->rope_base > 0.0)) return false;
     if ((c->k_cache == nullptr) != (c->v_cache == nullptr)) return false;
+    if (c->fused_projections != 0 && c->fused_projections != 1) return false;
     return true;
 }
 
@@ -240,6 +253,8 @@ extern "C" int dash_layer_workspace(const dash_layer_cfg* cfg, int64_t n, int S,
     off += kLtWorkspace;
     off += align_up(dash_workspace_bytes(DASH_WS_COMPACT, n, S, 0, 0, 0, cfg->dt), 256);
     off += align_up(dash_workspace_bytes(DASH_WS_ATTENTION, n, S, cfg->Hq, cfg->Hkv, cfg->D, cfg->dt), 256);
+    off += align_up((size_t)n * (cfg->D / 2) * sizeof(float2), 256);              // (cos, sin) of every row for the QKV epilogue
+    off += align_up((size_t)n * ((cfg->d + 255) / 256) * sizeof(float2), 256);    // per-row partial sums of the output-projection epilogue
     out->total = off;
     return DASH_OK;
 }
@@ -250,6 +265,7 @@ struct StepWs {
     dash_layer_ws_layout L;
     char *Hn, *QKV, *O, *U, *Ht, *lt_ws, *compact_ws, *attn_ws;
     size_t compact_bytes, attn_bytes;
+    float2 *rope_tab, *sums;
 };
 
 static int carve_ws(const dash_layer_cfg* cfg, int64_t n, int S, void* ws, StepWs* out) {
@@ -262,6 +278,8 @@ static int carve_ws(const dash_layer_cfg* cfg, int64_t n, int S, void* ws, StepW
     out->compact_bytes = align_up(dash_workspace_bytes(DASH_WS_COMPACT, n, S, 0, 0, 0, cfg->dt), 256);
     out->attn_ws = out->compact_ws + out->compact_bytes;
     out->attn_bytes = dash_workspace_bytes(DASH_WS_ATTENTION, n, S, cfg->Hq, cfg->Hkv, cfg->D, cfg->dt);
+    out->rope_tab = (float2*)(out->attn_ws + align_up(out->attn_bytes, 256));
+    out->sums = (float2*)((char*)out->rope_tab + align_up((size_t)n * (cfg->D / 2) * sizeof(float2), 256));
     return DASH_OK;
 }
 
@@ -274,10 +292,10 @@ static int launch_rmsnorm(dash_dtype dt, const void* X, const void* weight, void
     return DASH_OK;
 }
 
-// U = Attn(LN(H)) (Eq. 1) into W.U: RMSNorm -> Q | K | V projection -> rotary embedding -> causal attention over the packed
-// active set -> output projection
-static int attention_branch(const dash_layer_cfg* cfg, const void* H_in, const int32_t* pos_in, const int32_t* cu_in, int S, int64_t n,
-                            int64_t max_seqlen, const StepWs& W, cudaStream_t st) {
+// O = attention(rotary(LN(H) Wqkv)) into W.O: RMSNorm -> Q | K | V projection (rotary embedding in the GEMM epilogue when this
+// library's GEMM takes the shape, else a pass of its own) -> causal attention over the packed active set
+static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int32_t* pos_in, const int32_t* cu_in, int S, int64_t n,
+                          int64_t max_seqlen, const StepWs& W, cudaStream_t st) {
     const int es = cfg->dt == DASH_BF16 ? 2 : 4;
     const bool bf = cfg->dt == DASH_BF16;
     const int d = cfg->d, Hq = cfg->Hq, Hkv = cfg->Hkv, D = cfg->D;
@@ -286,17 +304,24 @@ static int attention_branch(const dash_layer_cfg* cfg, const void* H_in, const i
     int rc;
     // LN (read as RMSNorm)
     if ((rc = launch_rmsnorm(cfg->dt, H_in, cfg->rms_weight, W.Hn, n, d, cfg->rms_eps, n_dev, st)) != DASH_OK) return rc;
-    // Q | K | V = Hn Wqkv
-    if ((rc = gemm_rowmajor(cfg->dt, W.Hn, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, W.lt_ws, st)) != DASH_OK) return rc;
-    // rotary embedding on the Q and K heads
-    RopeFreq fr;
-    for (int i = 0; i < D / 2; ++i) fr.inv_freq[i] = pow(cfg->rope_base, -2.0 * i / D);
-    const int heads = Hq + Hkv;
-    if (bf && D == 128) rope_kernel<true, 128><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
-    else if (bf) rope_kernel<true, 64><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
-    else if (D == 128) rope_kernel<false, 128><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
-    else rope_kernel<false, 64><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
-    DASH_CUDA_TRY(cudaGetLastError());
+    GemmEpilogue e;
+    e.D = D; e.n_rot_cols = (Hq + Hkv) * D; e.rope_table = W.rope_tab;
+    if (bf && cfg->fused_projections && gemm_shape_ok(GEMM_ROPE, n, nq, d, d, nq, e)) {
+        // Q | K | V = Hn Wqkv, Q and K heads rotated on the accumulators
+        if ((rc = launch_rope_table(pos_in, n, D, cfg->rope_base, W.rope_tab, n_dev, st)) != DASH_OK) return rc;
+        if ((rc = gemm_bf16(GEMM_ROPE, W.Hn, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, e, n_dev, st)) != DASH_OK) return rc;
+    } else {
+        if ((rc = project(cfg->fused_projections != 0, cfg->dt, W.Hn, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, n_dev, W.lt_ws, st)) != DASH_OK) return rc;
+        // rotary embedding on the Q and K heads
+        RopeFreq fr;
+        for (int i = 0; i < D / 2; ++i) fr.inv_freq[i] = pow(cfg->rope_base, -2.0 * i / D);
+        const int heads = Hq + Hkv;
+        if (bf && D == 128) rope_kernel<true, 128><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
+        else if (bf) rope_kernel<true, 64><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
+        else if (D == 128) rope_kernel<false, 128><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
+        else rope_kernel<false, 64><<<rows_grid8(n), 256, 0, st>>>(W.QKV, nq * es, pos_in, n, heads, fr, n_dev);
+        DASH_CUDA_TRY(cudaGetLastError());
+    }
     if (cfg->k_cache) {
         // this depth's KV cache rows: keys (rotary applied) and values of the entering tokens, packed [n, Hkv, D]
         const int64_t kvb = (int64_t)Hkv * D * es;
@@ -304,12 +329,26 @@ static int attention_branch(const dash_layer_cfg* cfg, const void* H_in, const i
         if ((rc = dash_scatter(W.QKV + (int64_t)(Hq + Hkv) * D * es, n, kvb, nq * es, nullptr, nullptr, 2, n_dev, cfg->v_cache, kvb, st)) != DASH_OK) return rc;
     }
     // attention over the packed active set
-    rc = dash_varlen_attention(W.QKV, W.QKV + (int64_t)Hq * D * es, W.QKV + (int64_t)(Hq + Hkv) * D * es, W.O, nullptr, nq, nq, nq,
-                               (int64_t)Hq * D, cu_in, S, n, max_seqlen, Hq, Hkv, D, 1.0f / sqrtf((float)D), 1, cfg->dt,
-                               W.attn_ws, W.attn_bytes, st);
-    if (rc != DASH_OK) return rc;
-    // U = O Wo  (pre-residual attention output, Eq. 1)
-    return gemm_rowmajor(cfg->dt, W.O, (int64_t)Hq * D, cfg->Wo, d, W.U, d, n, d, (int64_t)Hq * D, W.lt_ws, st);
+    return dash_varlen_attention(W.QKV, W.QKV + (int64_t)Hq * D * es, W.QKV + (int64_t)(Hq + Hkv) * D * es, W.O, nullptr, nq, nq, nq,
+                                 (int64_t)Hq * D, cu_in, S, n, max_seqlen, Hq, Hkv, D, 1.0f / sqrtf((float)D), 1, cfg->dt,
+                                 W.attn_ws, W.attn_bytes, st);
+}
+
+// U = O Wo  (pre-residual attention output, Eq. 1) into W.U
+static int out_proj_U(const dash_layer_cfg* cfg, const int32_t* cu_in, int S, int64_t n, const StepWs& W, cudaStream_t st) {
+    const int64_t hd = (int64_t)cfg->Hq * cfg->D;
+    return project(cfg->fused_projections != 0, cfg->dt, W.O, hd, cfg->Wo, cfg->d, W.U, cfg->d, n, cfg->d, hd, cu_in + S, W.lt_ws, st);
+}
+
+// Output projection with the residual in its epilogue: dst[idx[row]] = H + O Wo (idx null: row), per-row sums of u^2, h^2 into W.sums.
+// Returns DASH_ERR_UNSUPPORTED when this library's GEMM does not take the shape (the caller then goes through U).
+static int out_proj_residual(const dash_layer_cfg* cfg, const void* H_in, const int32_t* idx, void* dst, const int32_t* cu_in, int S, int64_t n,
+                             const StepWs& W, cudaStream_t st) {
+    const int64_t hd = (int64_t)cfg->Hq * cfg->D;
+    GemmEpilogue e;
+    e.H = H_in; e.ldh = cfg->d; e.tok_index = idx; e.x_full = dst; e.ldx = cfg->d; e.sums = W.sums;
+    if (!cfg->fused_projections || cfg->dt != DASH_BF16 || !gemm_shape_ok(GEMM_RESID, n, cfg->d, hd, hd, cfg->d, e)) return DASH_ERR_UNSUPPORTED;
+    return gemm_bf16(GEMM_RESID, W.O, hd, cfg->Wo, cfg->d, nullptr, 0, n, cfg->d, hd, e, cu_in + S, st);
 }
 
 // r (and, threshold rule, the keep mask) from U and H, H~ = H + U into W.Ht; keep-count rule: the radix select on r
@@ -357,13 +396,23 @@ extern "C" int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, cons
         if (!aligned16(H_in) || !aligned16(x_full) || !aligned16(H_next) || !aligned16(cfg->Wqkv) || !aligned16(cfg->Wo) ||
             !aligned16(cfg->rms_weight))
             return DASH_ERR_INVALID_ARG;
-        if ((rc = attention_branch(cfg, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
+        if ((rc = attention_to_O(cfg, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
         if (cfg->sel_mode == DASH_SEL_THRESHOLD && cfg->scatter_which == 2) {
-            // r, H~ = H + U, the halting rule, the scatter of H~ and the compaction of the rows that stay, in one pass
-            return launch_delta_tail(W.U, H_in, nullptr, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau, cfg->keep_first,
+            // output projection with H~ = H + U written straight to x_full and the row sums of u^2, h^2 beside it; then the score, the
+            // halting rule and the compaction of the rows that stay (from x_full) in one pass
+            rc = out_proj_residual(cfg, H_in, tok_index_in, x_full, cu_in, S, n, W, st);
+            if (rc == DASH_OK)
+                return launch_delta_tail(nullptr, nullptr, nullptr, W.sums, d / 256, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau,
+                                         cfg->keep_first, cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out,
+                                         tok_index_next, pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, st);
+            if (rc != DASH_ERR_UNSUPPORTED) return rc;
+            // shapes this library's GEMM does not take: U through the library GEMM, then r, H~, the rule, scatter and compaction in one pass
+            if ((rc = out_proj_U(cfg, cu_in, S, n, W, st)) != DASH_OK) return rc;
+            return launch_delta_tail(W.U, H_in, nullptr, nullptr, 0, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau, cfg->keep_first,
                                      cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out, tok_index_next,
                                      pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, st);
         }
+        if ((rc = out_proj_U(cfg, cu_in, S, n, W, st)) != DASH_OK) return rc;
         if ((rc = score_and_select(cfg, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;
         // updated states reach the full-length output (halted tokens stay frozen there from now on)
         rc = dash_scatter(W.Ht, n, (int64_t)d * es, (int64_t)d * es, tok_index_in, mask_out, cfg->scatter_which, cu_in + S, x_full,
@@ -417,12 +466,31 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         return DASH_ERR_INVALID_ARG;
     const int32_t* n_dev = cu_in + S;
     // U = Attn(LN(H)); score and selection from U; H~ = H + U
-    if ((rc = attention_branch(a, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
-    if ((rc = score_and_select(a, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;   // also leaves H~ in W.Ht
+    if ((rc = attention_to_O(a, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
+    rc = cfg->signal == DASH_SIGNAL_ATTN ? out_proj_residual(a, H_in, nullptr, W.Ht, cu_in, S, n, W, st) : DASH_ERR_UNSUPPORTED;
+    if (rc == DASH_OK) {
+        // H~ came out of the projection's epilogue (into W.Ht) with the row sums: finish the score, then the rule
+        dash_threshold ft = {a->tau, a->keep_first, a->keep_last, cu_in, S, mask_out};
+        if ((rc = launch_sums_to_score(W.sums, d / 256, n, a->norm_mode, a->norm_eps, r_out, a->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr,
+                                       n_dev, st)) != DASH_OK) return rc;
+        if (a->sel_mode != DASH_SEL_THRESHOLD &&
+            (rc = dash_select(r_out, n, cu_in, S, a->sel_mode, a->tau, a->keep_counts, a->keep_first, a->keep_last, mask_out, nullptr, 0, st)) != DASH_OK)
+            return rc;
+    } else if (rc == DASH_ERR_UNSUPPORTED) {
+        if ((rc = out_proj_U(a, cu_in, S, n, W, st)) != DASH_OK) return rc;
+        if ((rc = score_and_select(a, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;   // also leaves H~ in W.Ht
+    } else {
+        return rc;
+    }
     // F = FFN(LN(H~)): gate | up projection, silu(gate) * up, down projection
     if ((rc = launch_rmsnorm(a->dt, W.Ht, cfg->rms2_weight, W.Hn, n, d, a->rms_eps, n_dev, st)) != DASH_OK) return rc;
-    if ((rc = gemm_rowmajor(a->dt, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, GU, 2 * (int64_t)m, n, 2 * (int64_t)m, d, W.lt_ws, st)) != DASH_OK) return rc;
-    {
+    GemmEpilogue eg;
+    eg.m = m;
+    if (a->fused_projections && a->dt == DASH_BF16 && gemm_shape_ok(GEMM_SWIGLU, n, 2 * (int64_t)m, d, d, 2 * (int64_t)m, eg)) {
+        // gate | up projection with silu(gate) * up on the accumulators: the [n, 2m] intermediate is never stored
+        if ((rc = gemm_bf16(GEMM_SWIGLU, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, ACT, m, n, 2 * (int64_t)m, d, eg, n_dev, st)) != DASH_OK) return rc;
+    } else {
+        if ((rc = gemm_rowmajor(a->dt, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, GU, 2 * (int64_t)m, n, 2 * (int64_t)m, d, W.lt_ws, st)) != DASH_OK) return rc;
         const int64_t total = n * (int64_t)(m / (16 / es));
         int64_t blocks = (total + 255) / 256, cap = (int64_t)sm_count() * 16;
         if (blocks > cap) blocks = cap;
@@ -430,7 +498,7 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         else swiglu_kernel<false><<<(int)blocks, 256, 0, st>>>(GU, 2 * (int64_t)m * es, ACT, (int64_t)m * es, n, m, n_dev);
         DASH_CUDA_TRY(cudaGetLastError());
     }
-    if ((rc = gemm_rowmajor(a->dt, ACT, m, cfg->Wd, d, F, d, n, d, m, W.lt_ws, st)) != DASH_OK) return rc;
+    if ((rc = project(a->fused_projections != 0, a->dt, ACT, m, cfg->Wd, d, F, d, n, d, m, n_dev, W.lt_ws, st)) != DASH_OK) return rc;
     if (cfg->signal == DASH_SIGNAL_BLOCK) {
         // ablation: score = change over the whole block, H' - H = U + F (formed in the gate | up buffer, free by now)
         if ((rc = dash_delta_norm(F, W.U, n, d, d, d, a->dt, DASH_NORM_ABS, a->norm_eps, r_out, GU, d, nullptr, nullptr, n_dev, st)) != DASH_OK) return rc;
@@ -444,7 +512,7 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
     }
     // H' = H~ + F to x_full (every entering token: H' is also the last updated value of the tokens that halt here) and,
     // for the tokens that stay, to the next block's packed buffer -- one pass, keep decisions taken from mask_out
-    return launch_delta_tail(F, W.Ht, mask_out, n, d, a->dt, a->norm_mode, a->norm_eps, a->tau, a->keep_first, a->keep_last, cu_in, S,
+    return launch_delta_tail(F, W.Ht, mask_out, nullptr, 0, n, d, a->dt, a->norm_mode, a->norm_eps, a->tau, a->keep_first, a->keep_last, cu_in, S,
                              tok_index_in, pos_in, x_full, H_next, nullptr, nullptr, tok_index_next, pos_next, cu_next, n_next_dev,
                              W.compact_ws, W.compact_bytes, st);
 }

@@ -49,7 +49,7 @@ class LayerCfg(Structure):
                 ("Wqkv", c_void_p), ("Wo", c_void_p), ("rms_weight", c_void_p), ("rms_eps", c_float),
                 ("rope_base", c_double), ("norm_mode", c_int), ("norm_eps", c_float), ("sel_mode", c_int),
                 ("tau", c_float), ("keep_counts", c_void_p), ("keep_first", c_int), ("keep_last", c_int),
-                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p)]
+                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p), ("fused_projections", c_int)]
 
 
 class LayerWsLayout(Structure):
@@ -306,7 +306,7 @@ class Layer:
     """Device-resident weights and configuration of one block for dash_layer_step."""
 
     def __init__(self, shape, weights, device, norm_mode=NORM_REL, norm_eps=1e-12, sel_mode=SEL_THRESHOLD, tau=0.0,
-                 keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2):
+                 keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2, fused_projections=False):
         self.shape = shape
         self.Wqkv = torch.cat([weights["Wq"], weights["Wk"], weights["Wv"]], dim=1).contiguous().to(device)
         self.Wo = weights["Wo"].contiguous().to(device)
@@ -314,7 +314,7 @@ class Layer:
         self.keep_counts = keep_counts
         self.cfg = LayerCfg(shape.d, shape.Hq, shape.Hkv, shape.D, dtype_code(self.Wo), self.Wqkv.data_ptr(), self.Wo.data_ptr(),
                             self.rms_w.data_ptr(), shape.rms_eps, shape.rope_base, norm_mode, norm_eps, sel_mode, tau,
-                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None)
+                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None, int(bool(fused_projections)))
 
     def set_tau(self, tau: float):
         self.cfg.tau = float(tau)

@@ -53,8 +53,9 @@ def _weights(sh, seed):
     return W
 
 
+@pytest.mark.parametrize("fused", [False, True], ids=["library_gemms", "fused_projections"])
 @pytest.mark.parametrize("case", ["cfg1_fp32", "mini_bf16_varlen"])
-def test_block_step_matches_oracle_threshold(case):
+def test_block_step_matches_oracle_threshold(case, fused):
     if case == "cfg1_fp32":
         w = wl.config1(T=512, seed=31)
     else:
@@ -69,7 +70,7 @@ def test_block_step_matches_oracle_threshold(case):
     tau = oc.kth_largest(ref0["r"], K)
     ref = oc.block_step(H, W, w.cu, pos, sh, tau=tau)
 
-    block = dash.Block(sh, W, DEV, tau=tau)
+    block = dash.Block(sh, W, DEV, tau=tau, fused_projections=fused)
     b = BlockBuffers(block, T, S)
     x_full = torch.full((T, sh.d), 9.0, dtype=sh.dtype, device=DEV)
     tok = torch.arange(T, dtype=torch.int32, device=DEV)
@@ -90,14 +91,15 @@ def test_block_step_matches_oracle_threshold(case):
         assert_close_h1(b.H_next[:k].float().cpu().numpy(), ref["rows"][0], "H_next", bf)
 
 
-def test_block_step_keep_count_rule_with_protected_tokens():
+@pytest.mark.parametrize("fused", [False, True], ids=["library_gemms", "fused_projections"])
+def test_block_step_keep_count_rule_with_protected_tokens(fused):
     w = wl.config2(T=640, seed=33, shape=wl.MINI)
     sh, T = w.shape, w.T
     H, W = w.tensors["H"], _weights(sh, 33)
     pos = wl.positions(w.cu)
     K = oc.keep_count(T, 0.667, 64, 32, mode=1)                  # Appendix A: protected prefix / suffix
     kc = torch.tensor([K], dtype=torch.int32, device=DEV)
-    block = dash.Block(sh, W, DEV, sel_mode=dash.SEL_KEEP_COUNT, keep_counts=kc, keep_first=64, keep_last=32)
+    block = dash.Block(sh, W, DEV, sel_mode=dash.SEL_KEEP_COUNT, keep_counts=kc, keep_first=64, keep_last=32, fused_projections=fused)
     b = BlockBuffers(block, T, 1)
     x_full = torch.zeros(T, sh.d, dtype=sh.dtype, device=DEV)
     run_block(block, H.to(DEV), torch.arange(T, dtype=torch.int32, device=DEV), pos.to(DEV), w.cu.to(DEV), T, x_full, b)
@@ -110,14 +112,15 @@ def test_block_step_keep_count_rule_with_protected_tokens():
     assert torch.equal(b.H_next[:K].cpu(), x_full.cpu()[np.flatnonzero(mask)])
 
 
-def test_block_step_qwen_shape_sampled_rows():
+@pytest.mark.parametrize("fused", [False, True], ids=["library_gemms", "fused_projections"])
+def test_block_step_qwen_shape_sampled_rows(fused):
     w = wl.config2(T=2048, seed=34)
     sh, T = w.shape, w.T
     H, W = w.tensors["H"], _weights(sh, 34)
     pos = wl.positions(w.cu)
     rows = wl.sample_rows(w.cu, 40, seed=8).numpy()
     ref = oc.block_step(H, W, w.cu, pos, sh, attn_rows=rows)
-    block = dash.Block(sh, W, DEV, tau=0.0)
+    block = dash.Block(sh, W, DEV, tau=0.0, fused_projections=fused)
     b = BlockBuffers(block, T, 1)
     x_full = torch.zeros(T, sh.d, dtype=sh.dtype, device=DEV)
     tok = torch.arange(T, dtype=torch.int32, device=DEV)
