@@ -209,7 +209,7 @@ def setup_block_step(args, dash, dev, rank):
     es = torch.empty(0, dtype=sh.dtype).element_size()
     H_host, pos_host = _pin(w.tensors["H"]), _pin(wl.positions(w.cu))
     tok_host, cu_host = _pin(torch.arange(T, dtype=torch.int32)), _pin(w.cu)
-    layer = dash.Layer(sh, w.weights[0], dev, tau=0.0, fused_projections=args.fused_projections)
+    layer = dash.Layer(sh, w.weights[0], dev, tau=0.0, fused_projections=not args.library_gemms)
     B = StepBuffers(dash, layer, T, S, sh.d, sh.dtype, dev)
     H = torch.empty(T, sh.d, dtype=sh.dtype, device=dev)
     pos, tok = torch.empty(T, dtype=torch.int32, device=dev), torch.empty(T, dtype=torch.int32, device=dev)
@@ -295,9 +295,9 @@ def setup_block_step(args, dash, dev, rank):
     name = "configs[0]: single fp32 layer, hidden 256, 4 heads of 64" if args.workload == "cfg1" else "configs[1]: Qwen2.5-7B-shaped single layer, bf16"
     return {
         "workload": f"{name}, batch 1, seq {T}, threshold at the {int(w.rho * 100)}th percentile ({n_active} of {T} tokens stay active)",
-        "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 5,
-        "launch_note": "per step: rmsnorm, rope, attention plan, attention, fused tail (score + residual + threshold + scatter + compaction) "
-                       "(+2 cuBLASLt GEMMs and a memset that are not this library's kernels)",
+        "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 7,
+        "launch_note": "per step: rmsnorm, rope table, QKV GEMM (+ rotary), attention plan, attention, output GEMM (+ residual, score sums), "
+                       "tail (score + threshold + compaction) (+ a memset)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(*host_out),
         "extra": {"n_active_after": n_active, "tau": tau}, "e2e_pipeline": e2e_pipeline,
         "attn": (lambda: dash.dash_varlen_attention(Q, Kt, V, cu, T, O=Obuf, ws=attn_ws)), "attn_flops": attention_flops(w.cu.tolist(), sh.Hq, sh.D),
@@ -315,7 +315,7 @@ def setup_cascade(args, dash, dev, rank):
     w = wl.config3(T=T, seed=rank_seed(2, rank), n_layers=Lr)
     sh, S, es = w.shape, w.S, 2
     Ks = [dash.dash_keep_count(T, 1.0 - f) for f in w.fractions]
-    layers = [dash.Layer(sh, w.weights[l], dev, tau=0.0, fused_projections=args.fused_projections) for l in range(Lr)]
+    layers = [dash.Layer(sh, w.weights[l], dev, tau=0.0, fused_projections=not args.library_gemms) for l in range(Lr)]
     A, Bb = StepBuffers(dash, layers[0], T, S, sh.d, sh.dtype, dev), StepBuffers(dash, layers[0], T, S, sh.d, sh.dtype, dev)
     H_host, pos_host = _pin(w.tensors["H"]), _pin(wl.positions(w.cu))
     tok_host, cu_host = _pin(torch.arange(T, dtype=torch.int32)), _pin(w.cu)
@@ -375,8 +375,8 @@ def setup_cascade(args, dash, dev, rank):
     fl_all = sum(attention_flops([0, n], sh.Hq, sh.D) for n in n_in)
     return {
         "workload": f"configs[2]: cascade of {Lr} Qwen2.5-7B-shaped layers, bf16, batch 1, seq {T}, tokens entering the layers {n_in}, "
-                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 5 * Lr,
-        "launch_note": f"{Lr} block steps of 5 kernels each (+2 cuBLASLt GEMMs per block step)",
+                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 7 * Lr,
+        "launch_note": f"{Lr} block steps of 7 kernels each",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(x_full_h, tok_h, cu_h),
         "extra": {"tokens_entering_layers": n_in, "active_after_last": got, "attention_flops_per_step": fl_all,
                   "value_counts": "tokens entering each of the 8 layers, summed"},
@@ -469,7 +469,7 @@ def setup_stack(args, dash, dev, rank):
     Wt = dict(wl.layer_weights(sh, rank_seed(5, rank))); Wt.update(wl.ffn_weights(sh, rank_seed(5, rank)))
     K = dash.dash_keep_count(T, rho, 64, 32, 1)
     kc = torch.tensor([K], dtype=torch.int32, device=dev)
-    blk = dash.Block(sh, Wt, dev, tau=0.0, keep_first=64, keep_last=32, fused_projections=args.fused_projections)   # one set of weights (timing only)
+    blk = dash.Block(sh, Wt, dev, tau=0.0, keep_first=64, keep_last=32, fused_projections=not args.library_gemms)   # one set of weights (timing only)
     lay = dash.dash_block_workspace(blk, T, S)
     ws = dash.workspace(lay.total, dev)
     H_host, pos_host = _pin(wl.hidden_states(T, sh.d, rank_seed(5, rank), sh.dtype)), _pin(wl.positions(cu_h))
@@ -536,9 +536,9 @@ def setup_stack(args, dash, dev, rank):
     return {
         "workload": f"the paper's efficiency setting: {Lr} Qwen2.5-7B-shaped blocks with feed-forward, bf16, batch 1, seq {T}, single-shot selection "
                     f"at block {l_s}, compression ratio {rho}, first 64 / last 32 kept ({K} tokens stay); a step = the whole prefill",
-        "dtype": "bf16", "step": (lambda: prefill(True)), "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 7 * Lr + 1,
-        "launch_note": f"{Lr} block steps: rmsnorm x2, rope, attention plan, attention, score (+ select once), swiglu, fused tail "
-                       "(+4 cuBLASLt GEMMs and a memset per block)",
+        "dtype": "bf16", "step": (lambda: prefill(True)), "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 11 * Lr + 1,
+        "launch_note": f"{Lr} block steps: rmsnorm x2, rope table, 4 GEMMs (rotary / residual + sums / SwiGLU / plain), attention plan, attention, "
+                       "score from sums (+ select once), tail (+ a memset per block)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(x_h, tok_h), "extra": extra,
         "attn": (lambda: dash.dash_varlen_attention(Q, Kt, V, cu, T, O=Obuf, ws=attn_ws)), "attn_flops": attention_flops([0, T], sh.Hq, sh.D),
         "attn_name": f"attention_kernel<{sh.D}> (dense block, {T} tokens)",
@@ -713,7 +713,7 @@ def run_ours(args):
     cfg = {"workload": W["workload"], "tokens_per_step_per_gpu": tokens,
            "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write, then {L2_FLUSH_BYTES >> 20} MiB read)", "status_word": status}
     cfg.update(W["extra"])
-    cfg["projections"] = "this library's tcgen05 GEMMs with fused epilogues" if args.fused_projections else "library GEMMs (cuBLASLt)"
+    cfg["projections"] = "library GEMMs (cuBLASLt)" if args.library_gemms else "this library's tcgen05 GEMMs (CTA pairs) with fused epilogues"
     out = {
         "metric": METRIC, "value": whole_job_value(tokens, world, t_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": t_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -826,8 +826,8 @@ def main():
     ap.add_argument("--seq", type=int, default=None, help="tokens per sequence (cfg1: 1024, cfg2: 8192, cfg3: 32768)")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--fused-projections", action="store_true",
-                    help="block steps use this library's tcgen05 GEMMs with fused epilogues instead of the library GEMMs (the default)")
+    ap.add_argument("--library-gemms", action="store_true",
+                    help="block steps use the library GEMMs (cuBLASLt) for the projections instead of this library's tcgen05 GEMMs with fused epilogues")
     args = ap.parse_args()
     if args.seq is None:
         args.seq = {"cfg1": 1024, "cfg2": 8192, "cfg3": 32768}.get(args.workload, 8192)

@@ -219,12 +219,12 @@ typedef struct {
     int          scatter_which;    /* rows of H~ written to x_full: 0 halted, 2 all */
     void*        k_cache;          /* NULL, or [n, Hkv, D]: this block's keys (rotary applied) of the entering tokens, */
     void*        v_cache;          /* and values: the rows a decoding step attends over at this depth (both or neither) */
-    int          fused_projections; /* 0: projections are library GEMMs (cuBLASLt), rotary embedding, residual and score in passes of
-                                     * this library.  1: this library's tcgen05 GEMMs with that work on their accumulators (rotary
-                                     * embedding in the QKV projection; H~ and the score's row sums in the output projection; SwiGLU
-                                     * in the gate | up projection): one rounding less per value, no U / gate | up intermediates;
-                                     * bf16 with 256-column tiles only (other shapes fall back to 0).  Measured 3-6 % slower than 0
-                                     * over long runs under the power cap, which is why 0 is the default. */
+    int          fused_projections; /* 1 (what the binding sets by default): the projections run in this library's tcgen05 GEMMs
+                                     * (256 x 256 tiles on CTA pairs) with the work that follows them on the accumulators: rotary
+                                     * embedding in the QKV projection; H~ and the score's row sums in the output projection;
+                                     * SwiGLU in the gate | up projection -- one rounding less per value, no U and no gate | up
+                                     * intermediate.  bf16 with 256-column tiles; other shapes and fp32 fall back to 0.
+                                     * 0: library GEMMs (cuBLASLt), rotary embedding, residual and score in passes of this library. */
 } dash_layer_cfg;
 
 /* Byte offsets of the intermediates inside the workspace of dash_layer_step

@@ -5,8 +5,11 @@
 //   RESID  : U = O Wo is never stored: H~ = H + U goes straight to x_full[tok[row]], and the per-row partial sums of
 //            u^2 and h^2 of this tile's columns go to a small buffer (the score of Eq. 2 is finished from them)
 //   SWIGLU : one tile holds 128 gate and the matching 128 up columns: act = silu(g) * u      (FFN of Alg. 1)
-// One CTA per SM; tile 128 x 256, K in steps of 64 through a 4-stage TMA ring; warp 0 issues the loads, warp 1 the MMAs,
-// warps 2-5 read the accumulators (two TMEM buffers, so a tile's epilogue overlaps the next tile's MMAs).
+// One CTA per SM, in clusters of two: a pair computes a 256 x 256 tile with tcgen05.mma.cta_group::2 -- CTA r holds rows
+// 128 r .. of the A tile and columns 128 r .. of the W tile, so every SM loads only half of the W operand.  K in steps of 64
+// through a 6-stage TMA ring; warp 0 of each CTA issues its loads (their bytes are counted on the pair's even CTA), warp 1 of
+// the even CTA issues the MMAs and releases stages / hands over accumulators in both CTAs with multicast commits, warps 2-5
+// of each CTA read their 128 accumulator rows (two TMEM buffers, so a tile's epilogue overlaps the next tile's MMAs).
 #include <math.h>
 
 #include "common.cuh"
@@ -17,16 +20,31 @@ namespace dash {
 
 using namespace ptx;
 
-constexpr int kGM = 128, kGN = 256, kGK = 64, kGStages = 4;
-constexpr int kGABytes = kGM * kGK * 2, kGBBytes = kGK * kGN * 2, kGStageBytes = kGABytes + kGBBytes;
+constexpr int kGM = 128, kGN = 256, kGK = 64, kGStages = 6;      // kGM: rows per CTA (256 per pair)
+constexpr int kGABytes = kGM * kGK * 2, kGBBytes = kGK * (kGN / 2) * 2, kGStageBytes = kGABytes + kGBBytes;   // per CTA
 constexpr int kGThreads = 192;
 constexpr int kGGroupN = 16;                 // n tiles per group of the tile order
 constexpr long long kGWait = 4000000000LL;
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+constexpr uint32_t kPeerMask = 0xFEFFFFFFu;   // clears the CTA-rank bit of a shared::cluster address: the pair's even CTA
+
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// tiled load into this CTA's shared memory whose bytes are counted on the barrier of the pair's even CTA
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar & kPeerMask), "r"(c0), "r"(c1) : "memory");
+}
+// arrives, once every tcgen05 operation issued so far has completed, on the barrier at this offset in both CTAs of the pair
+__device__ __forceinline__ void commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void arrive_on_leader(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerMask) : "memory");
 }
 // The low word of a shared-memory descriptor holds the start address (>> 4) and the leading offset, the high word
 // everything that does not change inside a tile: stepping through a tile is a 32-bit add.
@@ -40,11 +58,11 @@ __device__ __forceinline__ void mma_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint32
                                           uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, {%7, %7, %7, %7, %7, %7, %7, %7}, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
 }
 
-// tile t -> (m tile, n tile): the n tiles come in groups of kGGroupN; within a group the m tiles run one after the other and
+// tile t -> (m tile of 256 rows, n tile): the n tiles come in groups of kGGroupN; within a group the m tiles run one after the other and
 // each visits the group's n tiles, so that the CTAs of a wave share a few A row-blocks and a few W column-blocks in L2
 __device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int& mt, int& nt) {
     const int per_group = m_tiles * kGGroupN;
@@ -64,7 +82,7 @@ struct GemmArgs {
 };
 
 template <int EPI>
-__global__ void __launch_bounds__(kGThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW, const GemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -76,59 +94,62 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const uint32_t slot = bars + 8 * (2 * kGStages + 4);
     volatile uint32_t* slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + (slot - smem_u32(smem_raw)));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rank = (int)cluster_rank();                  // 0: the pair's even CTA (issues the MMAs, owns the full / acc_empty barriers)
     if (warp == 1) {
         if (lane == 0) {
             for (int s = 0; s < kGStages; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
-            for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 128); }
+            for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 256); }
             fence_barrier_init();
             fence_proxy_async_smem();
         }
         __syncwarp();
-        tmem_alloc(slot, 512);
-        tmem_relinquish();
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     } else if (warp == 0 && lane == 0) {
         prefetch_tensormap(&mapA); prefetch_tensormap(&mapW);
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();                                    // the peer's barriers exist before anything is signalled across
     tc_fence_after();
     const uint32_t tmem = *slot_gen;
-    const int m_tiles = (g.n + kGM - 1) / kGM, n_tiles = g.n_tiles, tiles = m_tiles * n_tiles, ksteps = g.K / kGK;
-    constexpr uint32_t idesc = idesc_bf16_f32(kGM, kGN, false, true);
+    const int m_tiles = (g.n + 2 * kGM - 1) / (2 * kGM), n_tiles = g.n_tiles, tiles = m_tiles * n_tiles, ksteps = g.K / kGK;
+    const int n_pairs = (int)gridDim.x / 2, pair = (int)blockIdx.x / 2;
+    constexpr uint32_t idesc = idesc_bf16_f32(2 * kGM, kGN, false, true);
     constexpr uint32_t hi = smem_desc_hi_sw128(1024);
 
     if (warp == 0) {
-        // ---- loads: A tile 128 x 64 (K-major), W tile 64 x 256 as four 64-column chunks (N-major) ----
+        // ---- loads of this CTA: its 128 x 64 half of the A tile (K-major), its 64 x 128 half of the W tile as two 64-column chunks ----
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+            for (int t = pair; t < tiles && ok; t += n_pairs) {
                 int mt, nt;
                 tile_coords(t, m_tiles, n_tiles, mt, nt);
-                const int m0 = mt * kGM;
+                const int m0 = mt * 2 * kGM + rank * kGM;
                 for (int k = 0; k < ksteps && ok; ++k, ++it) {
                     const int s = it % kGStages;
                     if (it >= kGStages) ok = mbar_wait(empty(s), ((it / kGStages) - 1) & 1, kGWait);
                     if (!ok) break;
                     const uint32_t sA = base + s * kGStageBytes, sB = sA + kGABytes;
-                    mbar_arrive_expect_tx(full(s), kGStageBytes);
-                    tma_load_2d(sA, &mapA, full(s), k * kGK, m0);
+                    if (rank == 0) mbar_arrive_expect_tx(full(s), 2 * kGStageBytes);     // both CTAs' bytes land on this barrier
+                    tma_load_2d_pair(sA, &mapA, full(s), k * kGK, m0);
 #pragma unroll
-                    for (int c = 0; c < kGN / 64; ++c) {
-                        // SWIGLU: columns 0-127 of the tile are gate features nt * 128 .., columns 128-255 the same features of "up"
-                        const int col = (EPI == GEMM_SWIGLU) ? ((c < 2 ? 0 : g.e.m) + nt * 128 + (c & 1) * 64) : (nt * kGN + c * 64);
-                        tma_load_2d(sB + c * (kGK * 128), &mapW, full(s), col, k * kGK);
+                    for (int c = 0; c < kGN / 2 / 64; ++c) {
+                        // SWIGLU: columns 0-127 of the tile (the even CTA's half) are gate features nt * 128 .., columns 128-255 the same features of "up"
+                        const int col = (EPI == GEMM_SWIGLU) ? (rank * g.e.m + nt * 128 + c * 64) : (nt * kGN + rank * (kGN / 2) + c * 64);
+                        tma_load_2d_pair(sB + c * (kGK * 128), &mapW, full(s), col, k * kGK);
                     }
                 }
             }
             if (!ok) atomicExch(g.status, DASH_ERR_TIMEOUT);
         }
     } else if (warp == 1) {
-        // ---- MMAs: four 128 x 256 x 16 steps per stage into the tile's TMEM buffer ----
-        if (lane == 0) {
+        // ---- MMAs (even CTA only): four 256 x 256 x 16 steps per stage into the tile's TMEM buffer of both CTAs ----
+        if (lane == 0 && rank == 0) {
             uint32_t it = 0, tl = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++tl) {
+            for (int t = pair; t < tiles && ok; t += n_pairs, ++tl) {
                 const int b = tl & 1;
                 if (tl >= 2) ok = mbar_wait(acc_empty(b), ((tl >> 1) - 1) & 1, kGWait);
                 if (!ok) break;
@@ -144,9 +165,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 #pragma unroll
                     for (int kk = 0; kk < kGK / 16; ++kk)
                         mma_ss_lh(tD, a_lo + ((kk * 32) >> 4), hi, b_lo + ((kk * 2048) >> 4), hi, idesc, (k > 0) || (kk > 0));
-                    tc_commit(empty(s));
+                    commit_pair(empty(s));
                 }
-                tc_commit(acc_full(b));
+                commit_pair(acc_full(b));
             }
             if (!ok) atomicExch(g.status, DASH_ERR_TIMEOUT);
         }
@@ -158,14 +179,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         if (g.n_dev) { const int nd = *g.n_dev; if (nd < n_true) n_true = nd; }
         uint32_t tl = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++tl) {
+        for (int t = pair; t < tiles; t += n_pairs, ++tl) {
             const int b = tl & 1;
             int mt, nt;
             tile_coords(t, m_tiles, n_tiles, mt, nt);
             ok = mbar_wait(acc_full(b), (tl >> 1) & 1, kGWait);
             if (!ok) break;
             tc_fence_after();
-            const int row = mt * kGM + q * 32 + lane;
+            const int row = mt * 2 * kGM + rank * kGM + q * 32 + lane;
             const bool live = row < n_true;
             const uint32_t tD = tmem + b * kGN + lane_base;
             if (EPI == GEMM_PLAIN) {
@@ -270,13 +291,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 }
             }
             tc_fence_before();
-            mbar_arrive(acc_empty(b));
+            arrive_on_leader(acc_empty(b));
         }
         if (!ok && lane == 0) atomicExch(g.status, DASH_ERR_TIMEOUT);
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, 512); }
+    cluster_sync_all();                                    // nobody leaves while the peer may still signal its barriers or read its tiles
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
 }
 
 // (cos, sin) of pos[t] * base^(-2i/D) for i < D/2; angles formed and reduced in fp64 (positions reach 1e5 rad at i = 0)
@@ -315,10 +340,10 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mw, const GemmA
         if (cudaFuncSetAttribute(gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
         configured = true;
     }
-    const int tiles = ((g.n + kGM - 1) / kGM) * g.n_tiles;
-    int grid = sm_count();
-    if (grid > tiles) grid = tiles;
-    gemm_kernel<EPI><<<grid, kGThreads, smem, st>>>(ma, mw, g);
+    const int tiles = ((g.n + 2 * kGM - 1) / (2 * kGM)) * g.n_tiles;
+    int pairs = sm_count() / 2;
+    if (pairs > tiles) pairs = tiles;
+    gemm_kernel<EPI><<<2 * pairs, kGThreads, smem, st>>>(ma, mw, g);
     return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 

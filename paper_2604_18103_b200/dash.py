@@ -306,7 +306,7 @@ class Layer:
     """Device-resident weights and configuration of one block for dash_layer_step."""
 
     def __init__(self, shape, weights, device, norm_mode=NORM_REL, norm_eps=1e-12, sel_mode=SEL_THRESHOLD, tau=0.0,
-                 keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2, fused_projections=False):
+                 keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2, fused_projections=True):
         self.shape = shape
         self.Wqkv = torch.cat([weights["Wq"], weights["Wk"], weights["Wv"]], dim=1).contiguous().to(device)
         self.Wo = weights["Wo"].contiguous().to(device)
