@@ -295,9 +295,9 @@ def setup_block_step(args, dash, dev, rank):
     name = "configs[0]: single fp32 layer, hidden 256, 4 heads of 64" if args.workload == "cfg1" else "configs[1]: Qwen2.5-7B-shaped single layer, bf16"
     return {
         "workload": f"{name}, batch 1, seq {T}, threshold at the {int(w.rho * 100)}th percentile ({n_active} of {T} tokens stay active)",
-        "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 7,
-        "launch_note": "per step: rmsnorm, rope table, QKV GEMM (+ rotary), attention plan, attention, output GEMM (+ residual, score sums), "
-                       "tail (score + threshold + compaction) (+ a memset)",
+        "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 6,
+        "launch_note": "per step: row factors + rotary angles, QKV GEMM (norm factor + rotary on the accumulators), attention plan, attention, "
+                       "output GEMM (+ residual, score sums), tail (score + threshold + compaction) (+ a memset)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(*host_out),
         "extra": {"n_active_after": n_active, "tau": tau}, "e2e_pipeline": e2e_pipeline,
         "attn": (lambda: dash.dash_varlen_attention(Q, Kt, V, cu, T, O=Obuf, ws=attn_ws)), "attn_flops": attention_flops(w.cu.tolist(), sh.Hq, sh.D),
@@ -375,8 +375,8 @@ def setup_cascade(args, dash, dev, rank):
     fl_all = sum(attention_flops([0, n], sh.Hq, sh.D) for n in n_in)
     return {
         "workload": f"configs[2]: cascade of {Lr} Qwen2.5-7B-shaped layers, bf16, batch 1, seq {T}, tokens entering the layers {n_in}, "
-                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 7 * Lr,
-        "launch_note": f"{Lr} block steps of 7 kernels each",
+                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 6 * Lr,
+        "launch_note": f"{Lr} block steps of 6 kernels each",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(x_full_h, tok_h, cu_h),
         "extra": {"tokens_entering_layers": n_in, "active_after_last": got, "attention_flops_per_step": fl_all,
                   "value_counts": "tokens entering each of the 8 layers, summed"},
@@ -536,8 +536,8 @@ def setup_stack(args, dash, dev, rank):
     return {
         "workload": f"the paper's efficiency setting: {Lr} Qwen2.5-7B-shaped blocks with feed-forward, bf16, batch 1, seq {T}, single-shot selection "
                     f"at block {l_s}, compression ratio {rho}, first 64 / last 32 kept ({K} tokens stay); a step = the whole prefill",
-        "dtype": "bf16", "step": (lambda: prefill(True)), "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 11 * Lr + 1,
-        "launch_note": f"{Lr} block steps: rmsnorm x2, rope table, 4 GEMMs (rotary / residual + sums / SwiGLU / plain), attention plan, attention, "
+        "dtype": "bf16", "step": (lambda: prefill(True)), "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 9 * Lr + 1,
+        "launch_note": f"{Lr} block steps: row factors + rotary angles, 4 GEMMs (rotary / residual + sums / SwiGLU / plain), attention plan, attention, "
                        "score from sums (+ select once), tail (+ a memset per block)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(x_h, tok_h), "extra": extra,
         "attn": (lambda: dash.dash_varlen_attention(Q, Kt, V, cu, T, O=Obuf, ws=attn_ws)), "attn_flops": attention_flops([0, T], sh.Hq, sh.D),

@@ -225,6 +225,9 @@ typedef struct {
                                      * SwiGLU in the gate | up projection -- one rounding less per value, no U and no gate | up
                                      * intermediate.  bf16 with 256-column tiles; other shapes and fp32 fall back to 0.
                                      * 0: library GEMMs (cuBLASLt), rotary embedding, residual and score in passes of this library. */
+    int          rms_folded;       /* 1: the norm's weight is already in Wqkv (row i of Wqkv multiplied by rms_weight[i]; rms_weight
+                                    * may then be NULL): the norm costs no pass of its own -- one pass over H yields the row factors
+                                    * 1 / rms, which the projection applies to its accumulators.  Needs fused_projections. */
 } dash_layer_cfg;
 
 /* Byte offsets of the intermediates inside the workspace of dash_layer_step
@@ -265,6 +268,7 @@ typedef struct {
     const void*  Wd;               /* [m, d] */
     const void*  rms2_weight;      /* [d]: weight of the norm in front of the FFN (attn.rms_eps is used) */
     dash_signal  signal;           /* what the score measures */
+    int          rms2_folded;      /* as attn.rms_folded, for the norm in front of the FFN and Wgu (needs DASH_SIGNAL_ATTN) */
 } dash_block_cfg;
 typedef struct {
     dash_layer_ws_layout attn;

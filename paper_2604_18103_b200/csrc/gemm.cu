@@ -3,7 +3,8 @@
 //   PLAIN  : C = A W                                                   (down projection of the FFN)
 //   ROPE   : Q | K | V = Hn Wqkv with the rotary embedding applied to the Q and K heads    (Eq. 1, inside Attn)
 //   RESID  : U = O Wo is never stored: H~ = H + U goes straight to x_full[tok[row]], and the per-row partial sums of
-//            u^2 and h^2 of this tile's columns go to a small buffer (the score of Eq. 2 is finished from them)
+//            u^2, h^2 and (h+u)^2 of this tile's columns go to a small buffer (the score of Eq. 2 and the next norm's row factor are
+//            finished from them)
 //   SWIGLU : one tile holds 128 gate and the matching 128 up columns: act = silu(g) * u      (FFN of Alg. 1)
 // One CTA per SM, in clusters of two: a pair computes a 256 x 256 tile with tcgen05.mma.cta_group::2 -- CTA r holds rows
 // 128 r .. of the A tile and columns 128 r .. of the W tile, so every SM loads only half of the W operand.  K in steps of 64
@@ -210,6 +211,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.C) + (int64_t)row * g.ldc + nt * kGN;
                 const int D = g.e.D, half = D >> 1;
                 const float2* cs = g.e.rope_table + (int64_t)row * half;       // (cos, sin) of this row
+                const float rsc = (g.e.row_scale && live) ? g.e.row_scale[row] : 1.0f;
                 for (int h0 = 0; h0 < kGN; h0 += D) {
                     const bool rotate = (nt * kGN + h0) < g.e.n_rot_cols;
                     // D = 128: two 32-column chunks per half; D = 64: one
@@ -222,7 +224,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                             float y1[32], y2[32];
 #pragma unroll
                             for (int e = 0; e < 32; ++e) {
-                                const float a = __uint_as_float(x1[e]), bb = __uint_as_float(x2[e]);
+                                const float a = __uint_as_float(x1[e]) * rsc, bb = __uint_as_float(x2[e]) * rsc;
                                 if (rotate) {
                                     const float2 t2 = cs[c + e];
                                     y1[e] = a * t2.x - bb * t2.y;
@@ -243,7 +245,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 // H~ = H + U (U in fp32, one rounding) to x_full[tok[row]]; sums of u^2 and h^2 over this tile's 256 columns
                 const __nv_bfloat16* hsrc = reinterpret_cast<const __nv_bfloat16*>(g.e.H) + (int64_t)row * g.e.ldh + nt * kGN;
                 __nv_bfloat16* dst = live ? reinterpret_cast<__nv_bfloat16*>(g.e.x_full) + (int64_t)(g.e.tok_index ? g.e.tok_index[row] : row) * g.e.ldx + nt * kGN : nullptr;
-                float su = 0.f, sh = 0.f;
+                float su = 0.f, sh = 0.f, st2 = 0.f;
 #pragma unroll
                 for (int c = 0; c < kGN / 32; ++c) {
                     uint32_t o[32];
@@ -261,15 +263,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                                 su += u * u;
                                 sh += hf[i] * hf[i];
                                 y[i] = hf[i] + u;
+                                st2 += y[i] * y[i];
                             }
                             st_v4(dst + c * 32 + e, make_uint4(pack_bf16(y[0], y[1]), pack_bf16(y[2], y[3]), pack_bf16(y[4], y[5]), pack_bf16(y[6], y[7])));
                         }
                     }
                 }
-                if (live) g.e.sums[(int64_t)row * n_tiles + nt] = make_float2(su, sh);
+                if (live) g.e.sums[(int64_t)row * n_tiles + nt] = make_float4(su, sh, st2, 0.f);
             } else {
                 // SWIGLU: columns 0-127 gate, 128-255 up of the same 128 features
                 __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.C) + (int64_t)row * g.ldc + nt * 128;
+                const float rsc = (g.e.row_scale && live) ? g.e.row_scale[row] : 1.0f;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t gt[32], up[32];
@@ -280,8 +284,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         float a[32];
 #pragma unroll
                         for (int e = 0; e < 32; ++e) {
-                            const float z = __uint_as_float(gt[e]);
-                            a[e] = z / (1.0f + __expf(-z)) * __uint_as_float(up[e]);
+                            const float z = __uint_as_float(gt[e]) * rsc;
+                            a[e] = z / (1.0f + __expf(-z)) * (__uint_as_float(up[e]) * rsc);
                         }
 #pragma unroll
                         for (int e = 0; e < 32; e += 8)
@@ -304,18 +308,43 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     }
 }
 
-// (cos, sin) of pos[t] * base^(-2i/D) for i < D/2; angles formed and reduced in fp64 (positions reach 1e5 rad at i = 0)
+// Per row (one warp): (cos, sin) of pos[t] * base^(-2i/D) for i < D/2, angles formed and reduced in fp64 (positions reach 1e5 rad
+// at i = 0); and, when asked, the row factor of the RMSNorm, 1 / sqrt(mean(h^2) + eps), from one pass over the bf16 row
 struct RopeFreqs { double inv_freq[64]; };
 __global__ void __launch_bounds__(256)
-rope_table_kernel(const int32_t* __restrict__ pos, int64_t n, int half, RopeFreqs fr, float2* __restrict__ table, const int32_t* __restrict__ n_dev) {
+row_prep_kernel(const int32_t* __restrict__ pos, int64_t n, int half, RopeFreqs fr, float2* __restrict__ table, const char* __restrict__ H,
+                int64_t ldh_b, int nvec, float inv_d, float eps, float* __restrict__ inv_rms, const int32_t* __restrict__ n_dev) {
     if (n_dev) { int64_t nd = *n_dev; if (nd < n) n = nd; }
-    const int64_t total = n * half;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t t = i / half;
-        const int k = (int)(i - t * half);
-        double sn, cs;
-        sincos((double)pos[t] * fr.inv_freq[k], &sn, &cs);
-        table[i] = make_float2((float)cs, (float)sn);
+    const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+    for (int64_t t = (int64_t)blockIdx.x * wpb + (threadIdx.x >> 5); t < n; t += (int64_t)gridDim.x * wpb) {
+        float ss = 0.f;
+        if (inv_rms) {
+            const char* h = H + t * ldh_b;
+            for (int base = 0; base < nvec; base += 128) {
+                uint4 x[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { const int v = base + k * 32 + lane; if (v < nvec) x[k] = ld_nc_v4(h + ((int64_t)v << 4)); }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int v = base + k * 32 + lane;
+                    if (v < nvec) {
+                        const float f[8] = {bf16lo(x[k].x), bf16hi(x[k].x), bf16lo(x[k].y), bf16hi(x[k].y), bf16lo(x[k].z), bf16hi(x[k].z), bf16lo(x[k].w), bf16hi(x[k].w)};
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) ss += f[e] * f[e];
+                    }
+                }
+            }
+        }
+        const double ps = (double)pos[t];
+        for (int i = lane; i < half; i += 32) {
+            double sn, cs;
+            sincos(ps * fr.inv_freq[i], &sn, &cs);
+            table[t * half + i] = make_float2((float)cs, (float)sn);
+        }
+        if (inv_rms) {
+            ss = warp_sum(ss);
+            if (lane == 0) inv_rms[t] = rsqrtf(ss * inv_d + eps);
+        }
     }
 }
 
@@ -377,14 +406,14 @@ int gemm_bf16(GemmEpilogueKind kind, const void* A, int64_t lda, const void* W, 
     }
 }
 
-int launch_rope_table(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const int32_t* n_dev, cudaStream_t st) {
+int launch_row_prep(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const void* H, int64_t ldh, int d, float rms_eps,
+                    float* inv_rms, const int32_t* n_dev, cudaStream_t st) {
     RopeFreqs fr;
     for (int i = 0; i < D / 2; ++i) fr.inv_freq[i] = pow(rope_base, -2.0 * i / D);
-    const int64_t total = n * (D / 2);
-    int64_t blocks = (total + 255) / 256, cap = (int64_t)sm_count() * 8;
+    int64_t blocks = (n + 7) / 8, cap = (int64_t)sm_count() * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    rope_table_kernel<<<(int)blocks, 256, 0, st>>>(pos, n, D / 2, fr, table, n_dev);
+    row_prep_kernel<<<(int)blocks, 256, 0, st>>>(pos, n, D / 2, fr, table, (const char*)H, ldh * 2, d * 2 / 16, 1.0f / d, rms_eps, inv_rms, n_dev);
     return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 

@@ -14,11 +14,15 @@ struct GemmEpilogue {
     // rope_table [n, D/2] = (cos, sin) of every row
     int D = 0, n_rot_cols = 0;
     const float2* rope_table = nullptr;
-    // RESID: x_full[tok_index[row]] (tok_index null: row) = H[row] + (A W)[row]; sums [n, N/256] = (sum u^2, sum h^2) per column tile
+    // ROPE, SWIGLU: row_scale (null: none) multiplies the accumulators of a row first -- 1 / rms(row) when the RMSNorm in front of the
+    // projection is folded into it (its weight into W, its row factor here)
+    const float* row_scale = nullptr;
+    // RESID: x_full[tok_index[row]] (tok_index null: row) = H[row] + (A W)[row]; sums [n, N/256] = (sum u^2, sum h^2, sum (h+u)^2, 0)
+    // per column tile
     const void* H = nullptr; int64_t ldh = 0;
     const int32_t* tok_index = nullptr;
     void* x_full = nullptr; int64_t ldx = 0;
-    float2* sums = nullptr;
+    float4* sums = nullptr;
     // SWIGLU: W = [K, 2m] (gate | up); C [n, m] = silu(A Wg) * (A Wu)
     int m = 0;
 };
@@ -28,6 +32,8 @@ bool gemm_shape_ok(GemmEpilogueKind kind, int64_t n, int64_t N, int64_t K, int64
 // C (or the epilogue's outputs) = A[n, K] W[K, N]; ld* in elements; n_dev: device true row count or null
 int gemm_bf16(GemmEpilogueKind kind, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc, int64_t n, int64_t N,
               int64_t K, const GemmEpilogue& e, const int32_t* n_dev, cudaStream_t st);
-int launch_rope_table(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const int32_t* n_dev, cudaStream_t st);
+// per row: (cos, sin) of pos * base^(-2i/D) into table [n, D/2]; with inv_rms non-null also 1 / sqrt(mean(H_row^2) + eps) (bf16 H, row stride ldh)
+int launch_row_prep(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const void* H, int64_t ldh, int d, float rms_eps,
+                    float* inv_rms, const int32_t* n_dev, cudaStream_t st);
 
 }  // namespace dash

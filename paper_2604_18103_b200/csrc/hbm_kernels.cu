@@ -439,7 +439,7 @@ __device__ __forceinline__ uint4 ld_cg_v4(const void* p) {
 struct TailArgs {
     const char* U; const char* H; int64_t ldU_b, ldH_b; int nvec; int mode; float eps;
     const uint8_t* mask_in;       // non-null: keep decisions are given (r and the mask are not formed), U is any update to add to H
-    const float2* sums; int n_sum_tiles;   // non-null: per-row partial (sum u^2, sum h^2) from the output-projection epilogue; with U null
+    const float4* sums; int n_sum_tiles;   // non-null: per-row partial (sum u^2, sum h^2, ..) from the output-projection epilogue; with U null
                                            // the rows are already in x_full and only the score, the decision and the compaction remain
     float tau; int keep_first, keep_last; const int32_t* cu_in; int S;
     const int32_t* tok_in; const int32_t* pos_in;
@@ -502,7 +502,7 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
                 if (a.sums) {
                     // the projection's column tiles, summed in a fixed order (lane i takes tiles i, i + 32, ...)
                     su = 0.f; sh = 0.f;
-                    for (int i = lane; i < a.n_sum_tiles; i += 32) { const float2 p2 = a.sums[(int64_t)row * a.n_sum_tiles + i]; su += p2.x; sh += p2.y; }
+                    for (int i = lane; i < a.n_sum_tiles; i += 32) { const float4 p2 = a.sums[(int64_t)row * a.n_sum_tiles + i]; su += p2.x; sh += p2.y; }
                 }
                 su = warp_sum(su);
                 sh = warp_sum(sh);
@@ -789,14 +789,17 @@ extern "C" int dash_compact_static(const uint8_t* mask, int64_t n, const int32_t
 namespace dash {
 size_t select_ws_bytes(int64_t, int) { return 256; }
 
-// r (and, with ft.mask_out set, the threshold decision) from the per-row partial sums of the output-projection epilogue
+// r (and, with ft.mask_out set, the threshold decision) from the per-row partial sums of the output-projection epilogue; with
+// inv_rms_out set also the row factor of the next RMSNorm, 1 / sqrt(mean((h+u)^2) + rms_eps)
 __global__ void __launch_bounds__(256)
-sums_to_score_kernel(const float2* __restrict__ sums, int n_sum_tiles, int64_t n, int mode, float eps, float* __restrict__ r_out,
-                     FusedThreshold ft, const int32_t* __restrict__ n_dev) {
+sums_to_score_kernel(const float4* __restrict__ sums, int n_sum_tiles, int64_t n, int mode, float eps, float* __restrict__ r_out,
+                     FusedThreshold ft, const int32_t* __restrict__ n_dev, float* __restrict__ inv_rms_out, float inv_d, float rms_eps) {
     if (n_dev) { int64_t nd = *n_dev; if (nd < n) n = nd; }
     for (int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; row < n; row += (int64_t)gridDim.x * blockDim.x) {
         float su = 0.f, sh = 0.f;
-        for (int i = 0; i < n_sum_tiles; ++i) { const float2 p2 = sums[row * n_sum_tiles + i]; su += p2.x; sh += p2.y; }
+        float st2 = 0.f;
+        for (int i = 0; i < n_sum_tiles; ++i) { const float4 p2 = sums[row * n_sum_tiles + i]; su += p2.x; sh += p2.y; st2 += p2.z; }
+        if (inv_rms_out) inv_rms_out[row] = rsqrtf(st2 * inv_d + rms_eps);
         const float num = sqrtf(su);
         const float r = (mode == DASH_NORM_ABS) ? num : num / fmaxf(sqrtf(sh), eps);
         r_out[row] = r;
@@ -809,20 +812,20 @@ sums_to_score_kernel(const float2* __restrict__ sums, int n_sum_tiles, int64_t n
     }
 }
 
-int launch_sums_to_score(const float2* sums, int n_sum_tiles, int64_t n, dash_norm_mode mode, float eps, float* r_out, const dash_threshold* fused,
-                         const int32_t* n_dev, cudaStream_t st) {
+int launch_sums_to_score(const float4* sums, int n_sum_tiles, int64_t n, dash_norm_mode mode, float eps, float* r_out, const dash_threshold* fused,
+                         const int32_t* n_dev, float* inv_rms_out, int d, float rms_eps, cudaStream_t st) {
     FusedThreshold ft = {0.f, 0, 0, nullptr, 0, nullptr};
     if (fused) ft = {fused->tau, fused->keep_first, fused->keep_last, fused->cu_seqlens, fused->S, fused->mask_out};
     int64_t blocks = (n + 255) / 256, cap = (int64_t)sm_count() * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    sums_to_score_kernel<<<(int)blocks, 256, 0, st>>>(sums, n_sum_tiles, n, (int)mode, eps, r_out, ft, n_dev);
+    sums_to_score_kernel<<<(int)blocks, 256, 0, st>>>(sums, n_sum_tiles, n, (int)mode, eps, r_out, ft, n_dev, inv_rms_out, 1.0f / d, rms_eps);
     return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 
 // Fused tail of the block step (see delta_tail_kernel).  Preconditions checked by the caller: threshold rule, every row
 // scattered, 16-byte aligned rows.  ws: the compaction workspace (ticket + one state word per 32-token tile).
-int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float2* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
+int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float4* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
                       int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st) {

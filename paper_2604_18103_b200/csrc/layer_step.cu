@@ -166,9 +166,9 @@ static int gemm_rowmajor(dash_dtype dt, const void* A, int64_t lda, const void* 
     return rc;
 }
 
-int launch_sums_to_score(const float2* sums, int n_sum_tiles, int64_t n, dash_norm_mode mode, float eps, float* r_out, const dash_threshold* fused,
-                         const int32_t* n_dev, cudaStream_t st);
-int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float2* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
+int launch_sums_to_score(const float4* sums, int n_sum_tiles, int64_t n, dash_norm_mode mode, float eps, float* r_out, const dash_threshold* fused,
+                         const int32_t* n_dev, float* inv_rms_out, int d, float rms_eps, cudaStream_t st);
+int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float4* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
                       int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st);
@@ -224,7 +224,8 @@ static bool cfg_ok(const dash_layer_cfg* c) {
     if (!c || c->d <= 0 || c->Hq < 1 || c->Hkv < 1 || (c->D != 64 && c->D != 128)) return false;
     if ((c->d % 8) || (c->Hq % c->Hkv)) return false;
     if (c->dt != DASH_F32 && c->dt != DASH_BF16) return false;
-    if (!c->Wqkv || !c->Wo || !c->rms_weight) return false;
+    if (!c->Wqkv || !c->Wo || (!c->rms_weight && !c->rms_folded)) return false;
+    if (c->rms_folded != 0 && c->rms_folded != 1) return false;
     if (c->sel_mode < DASH_SEL_THRESHOLD || c->sel_mode > DASH_SEL_KEEP_COUNT_HALT_HIGH) return false;
     if ((c->sel_mode == DASH_SEL_KEEP_COUNT || c->sel_mode == DASH_SEL_KEEP_COUNT_HALT_HIGH) && !c->keep_counts) return false;
     if (c->keep_first < 0 || c->keep_last < 0) return false;
@@ -254,7 +255,8 @@ extern "C" int dash_layer_workspace(const dash_layer_cfg* cfg, int64_t n, int S,
     off += align_up(dash_workspace_bytes(DASH_WS_COMPACT, n, S, 0, 0, 0, cfg->dt), 256);
     off += align_up(dash_workspace_bytes(DASH_WS_ATTENTION, n, S, cfg->Hq, cfg->Hkv, cfg->D, cfg->dt), 256);
     off += align_up((size_t)n * (cfg->D / 2) * sizeof(float2), 256);              // (cos, sin) of every row for the QKV epilogue
-    off += align_up((size_t)n * ((cfg->d + 255) / 256) * sizeof(float2), 256);    // per-row partial sums of the output-projection epilogue
+    off += align_up((size_t)n * ((cfg->d + 255) / 256) * sizeof(float4), 256);    // per-row partial sums of the output-projection epilogue
+    off += 2 * align_up((size_t)n * sizeof(float), 256);                          // row factors of the two folded norms
     out->total = off;
     return DASH_OK;
 }
@@ -265,7 +267,9 @@ struct StepWs {
     dash_layer_ws_layout L;
     char *Hn, *QKV, *O, *U, *Ht, *lt_ws, *compact_ws, *attn_ws;
     size_t compact_bytes, attn_bytes;
-    float2 *rope_tab, *sums;
+    float2* rope_tab;
+    float4* sums;
+    float *inv_rms, *inv_rms2;
 };
 
 static int carve_ws(const dash_layer_cfg* cfg, int64_t n, int S, void* ws, StepWs* out) {
@@ -279,7 +283,9 @@ static int carve_ws(const dash_layer_cfg* cfg, int64_t n, int S, void* ws, StepW
     out->attn_ws = out->compact_ws + out->compact_bytes;
     out->attn_bytes = dash_workspace_bytes(DASH_WS_ATTENTION, n, S, cfg->Hq, cfg->Hkv, cfg->D, cfg->dt);
     out->rope_tab = (float2*)(out->attn_ws + align_up(out->attn_bytes, 256));
-    out->sums = (float2*)((char*)out->rope_tab + align_up((size_t)n * (cfg->D / 2) * sizeof(float2), 256));
+    out->sums = (float4*)((char*)out->rope_tab + align_up((size_t)n * (cfg->D / 2) * sizeof(float2), 256));
+    out->inv_rms = (float*)((char*)out->sums + align_up((size_t)n * ((cfg->d + 255) / 256) * sizeof(float4), 256));
+    out->inv_rms2 = (float*)((char*)out->inv_rms + align_up((size_t)n * sizeof(float), 256));
     return DASH_OK;
 }
 
@@ -302,15 +308,23 @@ static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int
     const int64_t nq = (int64_t)(Hq + 2 * Hkv) * D;
     const int32_t* n_dev = cu_in + S;            // true number of entering tokens lives on the device
     int rc;
-    // LN (read as RMSNorm)
-    if ((rc = launch_rmsnorm(cfg->dt, H_in, cfg->rms_weight, W.Hn, n, d, cfg->rms_eps, n_dev, st)) != DASH_OK) return rc;
     GemmEpilogue e;
     e.D = D; e.n_rot_cols = (Hq + Hkv) * D; e.rope_table = W.rope_tab;
-    if (bf && cfg->fused_projections && gemm_shape_ok(GEMM_ROPE, n, nq, d, d, nq, e)) {
-        // Q | K | V = Hn Wqkv, Q and K heads rotated on the accumulators
-        if ((rc = launch_rope_table(pos_in, n, D, cfg->rope_base, W.rope_tab, n_dev, st)) != DASH_OK) return rc;
+    const bool fused = bf && cfg->fused_projections && gemm_shape_ok(GEMM_ROPE, n, nq, d, d, nq, e);
+    if (fused && cfg->rms_folded) {
+        // LN folded into the projection: its weight sits in Wqkv, its row factor 1 / rms is applied to the accumulators.
+        // One pass over H gives the row factors and the rotary angles; Q | K | V = (H Wqkv) / rms, Q and K rotated.
+        if ((rc = launch_row_prep(pos_in, n, D, cfg->rope_base, W.rope_tab, H_in, d, d, cfg->rms_eps, W.inv_rms, n_dev, st)) != DASH_OK) return rc;
+        e.row_scale = W.inv_rms;
+        if ((rc = gemm_bf16(GEMM_ROPE, H_in, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, e, n_dev, st)) != DASH_OK) return rc;
+    } else if (fused) {
+        // LN (read as RMSNorm), then Q | K | V = Hn Wqkv with the Q and K heads rotated on the accumulators
+        if ((rc = launch_rmsnorm(cfg->dt, H_in, cfg->rms_weight, W.Hn, n, d, cfg->rms_eps, n_dev, st)) != DASH_OK) return rc;
+        if ((rc = launch_row_prep(pos_in, n, D, cfg->rope_base, W.rope_tab, nullptr, 0, d, 0.f, nullptr, n_dev, st)) != DASH_OK) return rc;
         if ((rc = gemm_bf16(GEMM_ROPE, W.Hn, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, e, n_dev, st)) != DASH_OK) return rc;
     } else {
+        if (cfg->rms_folded) return DASH_ERR_UNSUPPORTED;      // folded weights need the fused projection (bf16, 256-column tiles)
+        if ((rc = launch_rmsnorm(cfg->dt, H_in, cfg->rms_weight, W.Hn, n, d, cfg->rms_eps, n_dev, st)) != DASH_OK) return rc;
         if ((rc = project(cfg->fused_projections != 0, cfg->dt, W.Hn, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, n_dev, W.lt_ws, st)) != DASH_OK) return rc;
         // rotary embedding on the Q and K heads
         RopeFreq fr;
@@ -368,7 +382,8 @@ static int score_and_select(const dash_layer_cfg* cfg, const void* H_in, const i
 static bool block_cfg_ok(const dash_block_cfg* c) {
     if (!c || !cfg_ok(&c->attn)) return false;
     const int epv = c->attn.dt == DASH_BF16 ? 8 : 4;
-    if (c->m <= 0 || (c->m % epv) || !c->Wgu || !c->Wd || !c->rms2_weight) return false;
+    if (c->m <= 0 || (c->m % epv) || !c->Wgu || !c->Wd || (!c->rms2_weight && !c->rms2_folded)) return false;
+    if (c->rms2_folded != 0 && c->rms2_folded != 1) return false;
     if (c->signal != DASH_SIGNAL_ATTN && c->signal != DASH_SIGNAL_BLOCK) return false;
     if (c->signal == DASH_SIGNAL_BLOCK && 2 * c->m < c->attn.d) return false;      // U + F is formed in the gate | up buffer
     return c->attn.scatter_which == 2;
@@ -394,7 +409,7 @@ extern "C" int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, cons
     const int d = cfg->d;
     if (n > 0) {
         if (!aligned16(H_in) || !aligned16(x_full) || !aligned16(H_next) || !aligned16(cfg->Wqkv) || !aligned16(cfg->Wo) ||
-            !aligned16(cfg->rms_weight))
+            (cfg->rms_weight && !aligned16(cfg->rms_weight)))
             return DASH_ERR_INVALID_ARG;
         if ((rc = attention_to_O(cfg, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
         if (cfg->sel_mode == DASH_SEL_THRESHOLD && cfg->scatter_which == 2) {
@@ -461,18 +476,20 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         return dash_compact(mask_out, 0, cu_in, S, nullptr, 0, pos_in, pos_next, tok_index_in, tok_index_next, nullptr, cu_next, n_next_dev,
                             W.compact_ws, W.compact_bytes, st);
     }
-    if (!aligned16(H_in) || !aligned16(x_full) || !aligned16(H_next) || !aligned16(a->Wqkv) || !aligned16(a->Wo) || !aligned16(a->rms_weight) ||
-        !aligned16(cfg->Wgu) || !aligned16(cfg->Wd) || !aligned16(cfg->rms2_weight))
+    if (!aligned16(H_in) || !aligned16(x_full) || !aligned16(H_next) || !aligned16(a->Wqkv) || !aligned16(a->Wo) || (a->rms_weight && !aligned16(a->rms_weight)) ||
+        !aligned16(cfg->Wgu) || !aligned16(cfg->Wd) || (cfg->rms2_weight && !aligned16(cfg->rms2_weight)))
         return DASH_ERR_INVALID_ARG;
     const int32_t* n_dev = cu_in + S;
     // U = Attn(LN(H)); score and selection from U; H~ = H + U
     if ((rc = attention_to_O(a, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
+    bool have_inv_rms2 = false;
     rc = cfg->signal == DASH_SIGNAL_ATTN ? out_proj_residual(a, H_in, nullptr, W.Ht, cu_in, S, n, W, st) : DASH_ERR_UNSUPPORTED;
     if (rc == DASH_OK) {
         // H~ came out of the projection's epilogue (into W.Ht) with the row sums: finish the score, then the rule
         dash_threshold ft = {a->tau, a->keep_first, a->keep_last, cu_in, S, mask_out};
+        have_inv_rms2 = cfg->rms2_folded != 0;
         if ((rc = launch_sums_to_score(W.sums, d / 256, n, a->norm_mode, a->norm_eps, r_out, a->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr,
-                                       n_dev, st)) != DASH_OK) return rc;
+                                       n_dev, have_inv_rms2 ? W.inv_rms2 : nullptr, d, a->rms_eps, st)) != DASH_OK) return rc;
         if (a->sel_mode != DASH_SEL_THRESHOLD &&
             (rc = dash_select(r_out, n, cu_in, S, a->sel_mode, a->tau, a->keep_counts, a->keep_first, a->keep_last, mask_out, nullptr, 0, st)) != DASH_OK)
             return rc;
@@ -483,12 +500,16 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         return rc;
     }
     // F = FFN(LN(H~)): gate | up projection, silu(gate) * up, down projection
-    if ((rc = launch_rmsnorm(a->dt, W.Ht, cfg->rms2_weight, W.Hn, n, d, a->rms_eps, n_dev, st)) != DASH_OK) return rc;
     GemmEpilogue eg;
     eg.m = m;
-    if (a->fused_projections && a->dt == DASH_BF16 && gemm_shape_ok(GEMM_SWIGLU, n, 2 * (int64_t)m, d, d, 2 * (int64_t)m, eg)) {
-        // gate | up projection with silu(gate) * up on the accumulators: the [n, 2m] intermediate is never stored
-        if ((rc = gemm_bf16(GEMM_SWIGLU, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, ACT, m, n, 2 * (int64_t)m, d, eg, n_dev, st)) != DASH_OK) return rc;
+    const bool fused_ffn = a->fused_projections && a->dt == DASH_BF16 && gemm_shape_ok(GEMM_SWIGLU, n, 2 * (int64_t)m, d, d, 2 * (int64_t)m, eg);
+    if (cfg->rms2_folded && !(fused_ffn && have_inv_rms2)) return DASH_ERR_UNSUPPORTED;   // folded weights need the fused projections
+    if (!cfg->rms2_folded && (rc = launch_rmsnorm(a->dt, W.Ht, cfg->rms2_weight, W.Hn, n, d, a->rms_eps, n_dev, st)) != DASH_OK) return rc;
+    if (fused_ffn) {
+        // gate | up projection with silu(gate) * up on the accumulators: the [n, 2m] intermediate is never stored; with the norm
+        // folded in, the operand is H~ itself and the accumulators take the row factor 1 / rms first
+        eg.row_scale = cfg->rms2_folded ? W.inv_rms2 : nullptr;
+        if ((rc = gemm_bf16(GEMM_SWIGLU, cfg->rms2_folded ? W.Ht : W.Hn, d, cfg->Wgu, 2 * (int64_t)m, ACT, m, n, 2 * (int64_t)m, d, eg, n_dev, st)) != DASH_OK) return rc;
     } else {
         if ((rc = gemm_rowmajor(a->dt, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, GU, 2 * (int64_t)m, n, 2 * (int64_t)m, d, W.lt_ws, st)) != DASH_OK) return rc;
         const int64_t total = n * (int64_t)(m / (16 / es));

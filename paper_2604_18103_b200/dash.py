@@ -49,7 +49,7 @@ class LayerCfg(Structure):
                 ("Wqkv", c_void_p), ("Wo", c_void_p), ("rms_weight", c_void_p), ("rms_eps", c_float),
                 ("rope_base", c_double), ("norm_mode", c_int), ("norm_eps", c_float), ("sel_mode", c_int),
                 ("tau", c_float), ("keep_counts", c_void_p), ("keep_first", c_int), ("keep_last", c_int),
-                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p), ("fused_projections", c_int)]
+                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p), ("fused_projections", c_int), ("rms_folded", c_int)]
 
 
 class LayerWsLayout(Structure):
@@ -58,7 +58,7 @@ class LayerWsLayout(Structure):
 
 
 class BlockCfg(Structure):
-    _fields_ = [("attn", LayerCfg), ("m", c_int), ("Wgu", c_void_p), ("Wd", c_void_p), ("rms2_weight", c_void_p), ("signal", c_int)]
+    _fields_ = [("attn", LayerCfg), ("m", c_int), ("Wgu", c_void_p), ("Wd", c_void_p), ("rms2_weight", c_void_p), ("signal", c_int), ("rms2_folded", c_int)]
 
 
 class BlockWsLayout(Structure):
@@ -302,19 +302,32 @@ def dash_decode_attention(q: torch.Tensor, Kc: torch.Tensor, Vc: torch.Tensor, c
 
 
 # ---- the block step ---------------------------------------------------------------
+def _projections_fit(shape) -> bool:
+    """True if this library's GEMMs take every projection of the block (256-column tiles, depth in steps of 64)."""
+    nq, hd = (shape.Hq + 2 * shape.Hkv) * shape.D, shape.Hq * shape.D
+    ok = shape.d % 256 == 0 and nq % 256 == 0 and ((shape.Hq + shape.Hkv) * shape.D) % 256 == 0 and hd % 64 == 0
+    return ok and (shape.m == 0 or shape.m % 128 == 0)
+
+
 class Layer:
     """Device-resident weights and configuration of one block for dash_layer_step."""
 
     def __init__(self, shape, weights, device, norm_mode=NORM_REL, norm_eps=1e-12, sel_mode=SEL_THRESHOLD, tau=0.0,
                  keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2, fused_projections=True):
         self.shape = shape
-        self.Wqkv = torch.cat([weights["Wq"], weights["Wk"], weights["Wv"]], dim=1).contiguous().to(device)
+        Wqkv = torch.cat([weights["Wq"], weights["Wk"], weights["Wv"]], dim=1)
+        # with fused projections (bf16) the norm's weight is folded into the projection once, here: the library then needs no
+        # normalisation pass (the row factor 1 / rms is applied to the projection's accumulators)
+        self.rms_folded = bool(fused_projections) and Wqkv.dtype == torch.bfloat16 and _projections_fit(shape)
+        if self.rms_folded:
+            Wqkv = (weights["rms_w"].float()[:, None] * Wqkv.float()).to(Wqkv.dtype)
+        self.Wqkv = Wqkv.contiguous().to(device)
         self.Wo = weights["Wo"].contiguous().to(device)
         self.rms_w = weights["rms_w"].contiguous().to(device)
         self.keep_counts = keep_counts
         self.cfg = LayerCfg(shape.d, shape.Hq, shape.Hkv, shape.D, dtype_code(self.Wo), self.Wqkv.data_ptr(), self.Wo.data_ptr(),
                             self.rms_w.data_ptr(), shape.rms_eps, shape.rope_base, norm_mode, norm_eps, sel_mode, tau,
-                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None, int(bool(fused_projections)))
+                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None, int(bool(fused_projections)), int(self.rms_folded))
 
     def set_tau(self, tau: float):
         self.cfg.tau = float(tau)
@@ -348,10 +361,14 @@ class Block:
     def __init__(self, shape, weights, device, signal=SIGNAL_ATTN, **layer_kwargs):
         self.layer = Layer(shape, weights, device, **layer_kwargs)
         self.shape = shape
-        self.Wgu = torch.cat([weights["Wg"], weights["Wu"]], dim=1).contiguous().to(device)
+        Wgu = torch.cat([weights["Wg"], weights["Wu"]], dim=1)
+        self.rms2_folded = self.layer.rms_folded and signal == SIGNAL_ATTN
+        if self.rms2_folded:
+            Wgu = (weights["rms2_w"].float()[:, None] * Wgu.float()).to(Wgu.dtype)
+        self.Wgu = Wgu.contiguous().to(device)
         self.Wd = weights["Wd"].contiguous().to(device)
         self.rms2_w = weights["rms2_w"].contiguous().to(device)
-        self.cfg = BlockCfg(self.layer.cfg, shape.m, self.Wgu.data_ptr(), self.Wd.data_ptr(), self.rms2_w.data_ptr(), signal)
+        self.cfg = BlockCfg(self.layer.cfg, shape.m, self.Wgu.data_ptr(), self.Wd.data_ptr(), self.rms2_w.data_ptr(), signal, int(self.rms2_folded))
 
     def set_tau(self, tau: float):
         self.cfg.attn.tau = float(tau)

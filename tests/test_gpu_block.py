@@ -50,6 +50,10 @@ def run_block(block, H, tok, pos, cu, max_seqlen, x_full, b):
 def _weights(sh, seed):
     W = dict(wl.layer_weights(sh, seed))
     W.update(wl.ffn_weights(sh, seed))
+    # norm weights that are not all ones: with fused projections the binding folds them into Wqkv and Wgu
+    g = torch.Generator().manual_seed(seed + 1000)
+    W["rms_w"] = (1.0 + 0.2 * torch.randn(sh.d, generator=g)).to(sh.dtype)
+    W["rms2_w"] = (1.0 + 0.2 * torch.randn(sh.d, generator=g)).to(sh.dtype)
     return W
 
 

@@ -62,7 +62,10 @@ def test_layer_step_matches_oracle(cfg, fused):
         w = wl.config2(T=900, seed=22, shape=wl.MINI)
         w.cu = wl.cu_from_lengths([300, 0, 471, 129])
     sh = w.shape
-    H, W = w.tensors["H"], w.weights[0]
+    H, W = w.tensors["H"], dict(w.weights[0])
+    if cfg != "cfg1":
+        # a norm weight that is not all ones: with fused projections the binding folds it into Wqkv
+        W["rms_w"] = (1.0 + 0.2 * torch.randn(sh.d, generator=torch.Generator().manual_seed(9))).to(sh.dtype)
     T, S = w.T, w.S
     pos = wl.positions(w.cu)
     ref0 = oc.layer_step(H, W, w.cu, pos, sh, tau=0.0)
@@ -88,7 +91,8 @@ def test_layer_step_matches_oracle(cfg, fused):
     if sh.dtype == torch.float32 or not fused:
         # with fused projections (bf16) the output projection adds the residual on its accumulators and U is never stored
         # (r and H~ below are what it leaves)
-        assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype).float().cpu().numpy(), ref["U"], "U")
+        # U is an intermediate too (stored after O was stored): twice the bar, as for Q and K above
+        assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype).float().cpu().numpy(), ref["U"], "U", tol=4e-2)
     # H~ of every entry token reaches x_full (threshold rule: score, residual, scatter and compaction run as one pass,
     # which writes H~ there and nowhere else); tok is the identity here
     assert_close_rms(x_full.float().cpu().numpy(), ref["Ht"], "H~ (x_full)")
