@@ -309,7 +309,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 }
 
 // Per row (one warp): (cos, sin) of pos[t] * base^(-2i/D) for i < D/2, angles formed and reduced in fp64 (positions reach 1e5 rad
-// at i = 0); and, when asked, the row factor of the RMSNorm, 1 / sqrt(mean(h^2) + eps), from one pass over the bf16 row
+// at i = 0: fp32 would lose the angle), evaluated in fp32 on the reduced angle; and, when asked, the row factor of the RMSNorm, 1 / sqrt(mean(h^2) + eps), from one pass over the bf16 row
 struct RopeFreqs { double inv_freq[64]; };
 __global__ void __launch_bounds__(256)
 row_prep_kernel(const int32_t* __restrict__ pos, int64_t n, int half, RopeFreqs fr, float2* __restrict__ table, const char* __restrict__ H,
@@ -337,9 +337,12 @@ row_prep_kernel(const int32_t* __restrict__ pos, int64_t n, int half, RopeFreqs 
         }
         const double ps = (double)pos[t];
         for (int i = lane; i < half; i += 32) {
-            double sn, cs;
-            sincos(ps * fr.inv_freq[i], &sn, &cs);
-            table[t * half + i] = make_float2((float)cs, (float)sn);
+            // angle formed and reduced to [-pi, pi] in fp64 (three operations), sine and cosine of the reduced angle in fp32
+            const double ang = ps * fr.inv_freq[i];
+            const double red = fma(-6.283185307179586476925286766559, rint(ang * 0.15915494309189533576888376337251), ang);
+            float sn, cs;
+            sincosf((float)red, &sn, &cs);
+            table[t * half + i] = make_float2(cs, sn);
         }
         if (inv_rms) {
             ss = warp_sum(ss);
