@@ -82,6 +82,7 @@ attention_plan_kernel(const int32_t* __restrict__ cu, int S, int Hq, int2* __res
     __shared__ int s_warp[33];
     __shared__ int s_max;
     const int tid = threadIdx.x;
+    pdl_launch_dependents();
     if (tid == 0) s_max = 0;
     __syncthreads();
     int mx = 0;
@@ -150,6 +151,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     volatile uint32_t* abort_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 68);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_launch_dependents();                               // the kernel behind may set itself up while this one drains
     volatile int* item_gen = reinterpret_cast<volatile int*>(smem_gen + L::kBars + 72);
 
     if (warp == 4) {
@@ -168,6 +170,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();                                            // set-up done; from here on the kernel in front (plan, projection) has completed
     const uint32_t tmem = *tmem_slot_gen;
     const uint32_t tS = tmem, tP = tmem, tO = tmem + 128;
 
@@ -441,19 +444,26 @@ static int launch_attention(const CUtensorMap& mq, const CUtensorMap& mk, const 
         if (cudaFuncSetAttribute(attention_kernel<D, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
         configured = true;
     }
-    attention_kernel<D, OUT_F32><<<grid, kAttnThreads, smem, st>>>(mq, mk, mv, p);
+    return launch_pdl(attention_kernel<D, OUT_F32>, grid, kAttnThreads, (size_t)smem, st, mq, mk, mv, p) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+}
+
+// The item list of a call (see attention_plan_kernel) into the head of its workspace.  A caller that knows cu_seqlens early
+// launches it ahead of the work that produces Q, K, V and then calls attention_planned().
+int attention_plan(const int32_t* cu_seqlens, int S, int64_t n, int Hq, void* ws, size_t ws_bytes, cudaStream_t st) {
+    if (!cu_seqlens || S < 1 || n < 0 || n > 0x7fffffffLL || Hq < 1) return DASH_ERR_INVALID_ARG;
+    if (n == 0) return DASH_OK;
+    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < 256 + plan_bytes(n, S)) return DASH_ERR_WORKSPACE;
+    if ((int64_t)plan_entries(n, S) * Hq > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
+    attention_plan_kernel<<<1, 1024, 0, st>>>(cu_seqlens, S, Hq, (int2*)((char*)ws + 256), (int*)((char*)ws + 4), (unsigned int*)ws,
+                                              (int64_t)plan_entries(n, S));
     return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 
-}  // namespace dash
-
-using namespace dash;
-
-extern "C" int dash_varlen_attention(const void* Q, const void* K, const void* V, void* O, float* lse,
-                                     int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
-                                     const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen,
-                                     int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
-                                     void* ws, size_t ws_bytes, void* stream) {
+static int attention_impl(const void* Q, const void* K, const void* V, void* O, float* lse,
+                          int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                          const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen,
+                          int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
+                          void* ws, size_t ws_bytes, void* stream, bool planned) {
     if (n < 0 || S < 1 || max_seqlen < 0 || Hq < 1 || Hkv < 1 || !cu_seqlens) return DASH_ERR_INVALID_ARG;
     if (dt != DASH_F32 && dt != DASH_BF16) return DASH_ERR_INVALID_ARG;
     if (D != 64 && D != 128) return DASH_ERR_UNSUPPORTED;
@@ -505,14 +515,29 @@ extern "C" int dash_varlen_attention(const void* Q, const void* K, const void* V
     p.ticket = (unsigned int*)ws;
     p.n_items = (const int*)((char*)ws + 4);
     p.plan = (const int2*)((char*)ws + 256);
-    if ((int64_t)plan_entries(n, S) * Hq > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
-    attention_plan_kernel<<<1, 1024, 0, st>>>(cu_seqlens, S, Hq, (int2*)((char*)ws + 256), (int*)((char*)ws + 4), (unsigned int*)ws,
-                                              (int64_t)plan_entries(n, S));
-    DASH_CUDA_TRY(cudaGetLastError());
+    if (!planned && (rc = attention_plan(cu_seqlens, S, n, Hq, ws, ws_bytes, st)) != DASH_OK) return rc;
     // persistent CTAs, two per SM, never more than there can be items
     int64_t grid64 = (int64_t)p.n_qtiles * Hq * S;
     if (grid64 > 2LL * sm_count()) grid64 = 2LL * sm_count();
     const int grid = (int)grid64;
     if (D == 128) return dt == DASH_F32 ? launch_attention<128, true>(mq, mk, mv, p, grid, st) : launch_attention<128, false>(mq, mk, mv, p, grid, st);
     return dt == DASH_F32 ? launch_attention<64, true>(mq, mk, mv, p, grid, st) : launch_attention<64, false>(mq, mk, mv, p, grid, st);
+}
+
+// same as dash_varlen_attention for a workspace whose item list attention_plan() has already been asked for on this stream
+int attention_planned(const void* Q, const void* K, const void* V, void* O, float* lse, int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                      const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen, int Hq, int Hkv, int D, float scale, dash_dtype dt,
+                      void* ws, size_t ws_bytes, cudaStream_t st) {
+    return attention_impl(Q, K, V, O, lse, ldq, ldk, ldv, ldo, cu_seqlens, S, n, max_seqlen, Hq, Hkv, D, scale, 1, dt, ws, ws_bytes, (void*)st, true);
+}
+
+}  // namespace dash
+
+extern "C" int dash_varlen_attention(const void* Q, const void* K, const void* V, void* O, float* lse,
+                                     int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                                     const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen,
+                                     int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
+                                     void* ws, size_t ws_bytes, void* stream) {
+    return dash::attention_impl(Q, K, V, O, lse, ldq, ldk, ldv, ldo, cu_seqlens, S, n, max_seqlen, Hq, Hkv, D, scale, causal, dt, ws, ws_bytes,
+                                stream, false);
 }

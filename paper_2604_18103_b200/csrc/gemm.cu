@@ -95,6 +95,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const uint32_t slot = bars + 8 * (2 * kGStages + 4);
     volatile uint32_t* slot_gen = reinterpret_cast<volatile uint32_t*>(smem_raw + (slot - smem_u32(smem_raw)));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // the kernel behind (attention, tail pass) may set itself up while this one drains; this kernel itself is launched in plain
+    // stream order: started early behind the attention or row kernels it measured 15 us slower per launch
+    pdl_launch_dependents();
     const int rank = (int)cluster_rank();                  // 0: the pair's even CTA (issues the MMAs, owns the full / acc_empty barriers)
     if (warp == 1) {
         if (lane == 0) {
@@ -314,6 +317,7 @@ struct RopeFreqs { double inv_freq[64]; };
 __global__ void __launch_bounds__(256)
 row_prep_kernel(const int32_t* __restrict__ pos, int64_t n, int half, RopeFreqs fr, float2* __restrict__ table, const char* __restrict__ H,
                 int64_t ldh_b, int nvec, float inv_d, float eps, float* __restrict__ inv_rms, const int32_t* __restrict__ n_dev) {
+    pdl_launch_dependents();
     if (n_dev) { int64_t nd = *n_dev; if (nd < n) n = nd; }
     const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
     for (int64_t t = (int64_t)blockIdx.x * wpb + (threadIdx.x >> 5); t < n; t += (int64_t)gridDim.x * wpb) {

@@ -1,6 +1,7 @@
 // HBM-bound kernels of the halted-prefill path: delta-attention score (+ fused
 // residual and threshold), halting rule, single-pass compaction, scatter.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace dash {
 
@@ -457,6 +458,7 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
     __shared__ int s_base, s_count;
     __shared__ unsigned int s_tile, s_ballot;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    ptx::pdl_wait();                                       // launched to start early: nothing global is touched before the kernel in front is done
     if (threadIdx.x == 0) s_tile = atomicAdd(a.ticket, 1u);
     __syncthreads();
     const int tile = (int)s_tile;
@@ -824,15 +826,23 @@ int launch_sums_to_score(const float4* sums, int n_sum_tiles, int64_t n, dash_no
 }
 
 // Fused tail of the block step (see delta_tail_kernel).  Preconditions checked by the caller: threshold rule, every row
-// scattered, 16-byte aligned rows.  ws: the compaction workspace (ticket + one state word per 32-token tile).
+// scattered, 16-byte aligned rows.  ws: the compaction workspace (ticket + one state word per 32-token tile); ws_is_clear: the
+// caller has already zeroed it on this stream with clear_tail_ws (ahead of the kernels in front, so that this launch follows a
+// kernel directly and may start while that one drains).
+static size_t tail_ws_clear_bytes(int64_t n) { return 256 + (size_t)((n + 31) / 32 > 0 ? (n + 31) / 32 : 1) * 8; }
+int clear_tail_ws(void* ws, size_t ws_bytes, int64_t n, cudaStream_t st) {
+    if (!ws || ((uintptr_t)ws % 256) || ws_bytes < compact_ws_bytes(n)) return DASH_ERR_WORKSPACE;
+    DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, tail_ws_clear_bytes(n), st));
+    return DASH_OK;
+}
 int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float4* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
-                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st) {
+                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, bool ws_is_clear, cudaStream_t st) {
     const int es = dt == DASH_BF16 ? 2 : 4;
     if (!ws || ((uintptr_t)ws % 256) || ws_bytes < compact_ws_bytes(n)) return DASH_ERR_WORKSPACE;
     const int tiles = (int)((n + 31) / 32) > 0 ? (int)((n + 31) / 32) : 1;
-    DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)tiles * 8, st));
+    if (!ws_is_clear) DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, tail_ws_clear_bytes(n), st));
     TailArgs a;
     a.mask_in = mask_in; a.sums = sums; a.n_sum_tiles = n_sum_tiles;
     a.U = (const char*)U; a.H = (const char*)H; a.ldU_b = a.ldH_b = (int64_t)d * es; a.nvec = d * es / 16; a.mode = (int)mode; a.eps = eps;
@@ -842,9 +852,8 @@ int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, cons
     a.ticket = (unsigned int*)ws; a.tile_state = (unsigned long long*)((char*)ws + 256);
     a.status = status_word_ptr();
     if (!a.status) return DASH_ERR_CUDA;
-    if (dt == DASH_BF16) delta_tail_kernel<true><<<tiles, kCompactThreads, 0, st>>>(a, n);
-    else delta_tail_kernel<false><<<tiles, kCompactThreads, 0, st>>>(a, n);
-    DASH_CUDA_TRY(cudaGetLastError());
+    if (dt == DASH_BF16) DASH_CUDA_TRY(launch_pdl(delta_tail_kernel<true>, tiles, kCompactThreads, 0, st, a, n));
+    else DASH_CUDA_TRY(launch_pdl(delta_tail_kernel<false>, tiles, kCompactThreads, 0, st, a, n));
     return DASH_OK;
 }
 size_t compact_ws_bytes_pub(int64_t n) { return compact_ws_bytes(n); }

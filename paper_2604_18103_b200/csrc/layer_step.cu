@@ -171,7 +171,12 @@ int launch_sums_to_score(const float4* sums, int n_sum_tiles, int64_t n, dash_no
 int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float4* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
-                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, cudaStream_t st);
+                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, bool ws_is_clear, cudaStream_t st);
+int clear_tail_ws(void* ws, size_t ws_bytes, int64_t n, cudaStream_t st);
+int attention_plan(const int32_t* cu_seqlens, int S, int64_t n, int Hq, void* ws, size_t ws_bytes, cudaStream_t st);
+int attention_planned(const void* Q, const void* K, const void* V, void* O, float* lse, int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                      const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen, int Hq, int Hkv, int D, float scale, dash_dtype dt,
+                      void* ws, size_t ws_bytes, cudaStream_t st);
 
 // C = A W: this library's GEMM when it takes the problem (bf16, 256-column tiles), the library GEMM otherwise
 static int project(bool own, dash_dtype dt, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc, int64_t n, int64_t N, int64_t K,
@@ -308,6 +313,9 @@ static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int
     const int64_t nq = (int64_t)(Hq + 2 * Hkv) * D;
     const int32_t* n_dev = cu_in + S;            // true number of entering tokens lives on the device
     int rc;
+    // the attention kernel's item list needs only cu_seqlens: asked for first, so that the attention kernel directly follows the
+    // projection in the stream (and may set itself up while that one drains)
+    if ((rc = attention_plan(cu_in, S, n, Hq, W.attn_ws, W.attn_bytes, st)) != DASH_OK) return rc;
     GemmEpilogue e;
     e.D = D; e.n_rot_cols = (Hq + Hkv) * D; e.rope_table = W.rope_tab;
     const bool fused = bf && cfg->fused_projections && gemm_shape_ok(GEMM_ROPE, n, nq, d, d, nq, e);
@@ -343,9 +351,9 @@ static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int
         if ((rc = dash_scatter(W.QKV + (int64_t)(Hq + Hkv) * D * es, n, kvb, nq * es, nullptr, nullptr, 2, n_dev, cfg->v_cache, kvb, st)) != DASH_OK) return rc;
     }
     // attention over the packed active set
-    return dash_varlen_attention(W.QKV, W.QKV + (int64_t)Hq * D * es, W.QKV + (int64_t)(Hq + Hkv) * D * es, W.O, nullptr, nq, nq, nq,
-                                 (int64_t)Hq * D, cu_in, S, n, max_seqlen, Hq, Hkv, D, 1.0f / sqrtf((float)D), 1, cfg->dt,
-                                 W.attn_ws, W.attn_bytes, st);
+    return attention_planned(W.QKV, W.QKV + (int64_t)Hq * D * es, W.QKV + (int64_t)(Hq + Hkv) * D * es, W.O, nullptr, nq, nq, nq,
+                             (int64_t)Hq * D, cu_in, S, n, max_seqlen, Hq, Hkv, D, 1.0f / sqrtf((float)D), cfg->dt,
+                             W.attn_ws, W.attn_bytes, st);
 }
 
 // U = O Wo  (pre-residual attention output, Eq. 1) into W.U
@@ -411,21 +419,24 @@ extern "C" int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, cons
         if (!aligned16(H_in) || !aligned16(x_full) || !aligned16(H_next) || !aligned16(cfg->Wqkv) || !aligned16(cfg->Wo) ||
             (cfg->rms_weight && !aligned16(cfg->rms_weight)))
             return DASH_ERR_INVALID_ARG;
+        const bool tail_pass = cfg->sel_mode == DASH_SEL_THRESHOLD && cfg->scatter_which == 2;
+        // the tail pass's look-back words are cleared up front: its launch then follows the output projection directly
+        if (tail_pass && (rc = clear_tail_ws(W.compact_ws, W.compact_bytes, n, st)) != DASH_OK) return rc;
         if ((rc = attention_to_O(cfg, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
-        if (cfg->sel_mode == DASH_SEL_THRESHOLD && cfg->scatter_which == 2) {
+        if (tail_pass) {
             // output projection with H~ = H + U written straight to x_full and the row sums of u^2, h^2 beside it; then the score, the
             // halting rule and the compaction of the rows that stay (from x_full) in one pass
             rc = out_proj_residual(cfg, H_in, tok_index_in, x_full, cu_in, S, n, W, st);
             if (rc == DASH_OK)
                 return launch_delta_tail(nullptr, nullptr, nullptr, W.sums, d / 256, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau,
                                          cfg->keep_first, cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out,
-                                         tok_index_next, pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, st);
+                                         tok_index_next, pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, true, st);
             if (rc != DASH_ERR_UNSUPPORTED) return rc;
             // shapes this library's GEMM does not take: U through the library GEMM, then r, H~, the rule, scatter and compaction in one pass
             if ((rc = out_proj_U(cfg, cu_in, S, n, W, st)) != DASH_OK) return rc;
             return launch_delta_tail(W.U, H_in, nullptr, nullptr, 0, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau, cfg->keep_first,
                                      cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out, tok_index_next,
-                                     pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, st);
+                                     pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, true, st);
         }
         if ((rc = out_proj_U(cfg, cu_in, S, n, W, st)) != DASH_OK) return rc;
         if ((rc = score_and_select(cfg, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;
@@ -480,6 +491,8 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         !aligned16(cfg->Wgu) || !aligned16(cfg->Wd) || (cfg->rms2_weight && !aligned16(cfg->rms2_weight)))
         return DASH_ERR_INVALID_ARG;
     const int32_t* n_dev = cu_in + S;
+    // the tail pass's look-back words are cleared up front: its launch then follows the down projection directly
+    if ((rc = clear_tail_ws(W.compact_ws, W.compact_bytes, n, st)) != DASH_OK) return rc;
     // U = Attn(LN(H)); score and selection from U; H~ = H + U
     if ((rc = attention_to_O(a, H_in, pos_in, cu_in, S, n, max_seqlen, W, st)) != DASH_OK) return rc;
     bool have_inv_rms2 = false;
@@ -535,5 +548,5 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
     // for the tokens that stay, to the next block's packed buffer -- one pass, keep decisions taken from mask_out
     return launch_delta_tail(F, W.Ht, mask_out, nullptr, 0, n, d, a->dt, a->norm_mode, a->norm_eps, a->tau, a->keep_first, a->keep_last, cu_in, S,
                              tok_index_in, pos_in, x_full, H_next, nullptr, nullptr, tok_index_next, pos_next, cu_next, n_next_dev,
-                             W.compact_ws, W.compact_bytes, st);
+                             W.compact_ws, W.compact_bytes, true, st);
 }

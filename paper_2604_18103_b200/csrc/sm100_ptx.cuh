@@ -172,6 +172,14 @@ __device__ __forceinline__ void tmem_st16x128_x8(uint32_t taddr, const uint32_t*
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Programmatic dependent launch.  A kernel launched with the stream-serialization attribute (launch_pdl) may be placed on an SM
+// while the kernel in front of it in the stream still runs: whatever it does before pdl_wait() -- barrier and TMEM set-up,
+// descriptor prefetch -- overlaps that kernel's tail; pdl_wait() returns once the kernel in front has completed and its writes
+// are visible (at once when there is none, or when the launch carried no attribute).  No global memory may be touched before it.
+// pdl_launch_dependents() lets the kernel behind start that early: once every CTA of this grid has executed it (or has exited).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
