@@ -4,7 +4,7 @@
 // head form the (mostly empty) 128-row operand of the tcgen05 MMAs, so K and V tiles stream through
 // shared memory once per KV head; the keys of a sequence are split over persistent CTAs (flash-decoding),
 // whose partial (max, sum, O) results a small merge kernel combines.
-//   plan kernel   : items (sequence, KV head, key-block range), sized so that about four items exist per SM
+//   plan kernel   : items (sequence, KV head, key-block range), sized so that one item exists per CTA (batches of up to 32 sequences: the CTAs plan for themselves) or four per SM (handed out by ticket)
 //   decode kernel : per item  S = Q K_j^T -> masked online softmax (one warp: the rows that exist) -> O += P V_j
 //   merge kernel  : O = sum_i 2^((m_i - m) c) O_i / sum_i 2^((m_i - m) c) l_i
 #include <math.h>
@@ -40,36 +40,63 @@ struct DecParams {
 // length and its items (item i -> CTA i mod grid; the items are equally long) from cu_seqlens itself, and so does the merge.
 constexpr int kSelfPlanSeqs = 32;
 __device__ __forceinline__ int dec_blocks(const int32_t* cu, int s) { return (cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN; }
-__device__ __forceinline__ int self_plan_chunk(const int32_t* cu, int S, int Hkv, int target) {
-    long long all = 0;
-    for (int s = 0; s < S; ++s) all += dec_blocks(cu, s);
-    all *= Hkv;
-    const long long chunk = (all + target - 1) / target;
-    return (int)(chunk < 1 ? 1 : chunk);
-}
-__device__ __forceinline__ int self_plan_count(const int32_t* cu, int S, int Hkv, int chunk) {
+// The plan of a self-planning launch, built once per CTA in shared memory: thread s fetches sequence s, thread 0 does the few
+// serial steps over at most kSelfPlanSeqs numbers.  (Every thread deriving it on its own from cu_seqlens cost the merge kernel of a
+// 32-sequence batch more than its merging.)
+struct SelfPlan {
+    int nb[kSelfPlanSeqs];        // key blocks of sequence s
+    int first[kSelfPlanSeqs];     // first item of sequence s (its Hkv heads follow each other, `per` items each)
+    int per[kSelfPlanSeqs];       // items per (sequence, KV head)
+    int chunk, n_items;
+};
+__device__ __forceinline__ int self_plan_count(const SelfPlan& sp, int S, int Hkv, int chunk) {
     int k = 0;
-    for (int s = 0; s < S; ++s) k += ((dec_blocks(cu, s) + chunk - 1) / chunk) * Hkv;
+    for (int s = 0; s < S; ++s) k += ((sp.nb[s] + chunk - 1) / chunk) * Hkv;
     return k;
 }
-__device__ __forceinline__ DecItem self_plan_item(const int32_t* cu, int S, int Hkv, int chunk, int item) {
+// Called by all threads of the CTA (it synchronises).  `target` is twice the number of CTAs.  Chunk length (key blocks per item):
+// preferred is one item per CTA -- the shortest chunk with at most target / 2 items (the last chunk of every sequence and head is an
+// item of its own, so the first guess can overshoot, and a CTA with a second item would double the kernel's time); half the pipeline
+// ramps and half the partial results to merge.  Taken when it keeps at least 17 of 20 CTAs busy; otherwise about `target` items.
+__device__ __forceinline__ void self_plan_build(SelfPlan& sp, const int32_t* cu, int S, int Hkv, int target) {
+    if ((int)threadIdx.x < S) sp.nb[threadIdx.x] = dec_blocks(cu, (int)threadIdx.x);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long all = 0;
+        for (int s = 0; s < S; ++s) all += sp.nb[s];
+        all *= Hkv;
+        long long chunk = (all + target - 1) / target;
+        if (chunk < 1) chunk = 1;
+        const int ctas = target / 2;
+        if (ctas > 0) {
+            long long c1 = (all + ctas - 1) / ctas;
+            if (c1 < 1) c1 = 1;
+            int cnt = self_plan_count(sp, S, Hkv, (int)c1);
+            for (int tries = 0; tries < 8 && cnt > ctas; ++tries) cnt = self_plan_count(sp, S, Hkv, (int)++c1);
+            if (cnt <= ctas && cnt * 20 >= ctas * 17) chunk = c1;
+        }
+        int k = 0;
+        for (int s = 0; s < S; ++s) {
+            sp.first[s] = k;
+            sp.per[s] = (sp.nb[s] + (int)chunk - 1) / (int)chunk;
+            k += sp.per[s] * Hkv;
+        }
+        sp.chunk = (int)chunk;
+        sp.n_items = k;
+    }
+    __syncthreads();
+}
+__device__ __forceinline__ DecItem self_plan_item(const SelfPlan& sp, int S, int Hkv, int item) {
     DecItem it = {0, 0, 0, 0};
     for (int s = 0; s < S; ++s) {
-        const int nb = dec_blocks(cu, s), per = (nb + chunk - 1) / chunk;
-        if (item < per * Hkv) {
-            const int h = item / per, i = item - h * per;
-            it.s = s; it.kvh = h; it.b0 = i * chunk; it.b1 = min((i + 1) * chunk, nb);
+        const int per = sp.per[s];
+        if (item < sp.first[s] + per * Hkv) {
+            const int r = item - sp.first[s], h = r / per, i = r - h * per;
+            it.s = s; it.kvh = h; it.b0 = i * sp.chunk; it.b1 = min((i + 1) * sp.chunk, sp.nb[s]);
             return it;
         }
-        item -= per * Hkv;
     }
     return it;
-}
-__device__ __forceinline__ int2 self_plan_segment(const int32_t* cu, int S, int Hkv, int chunk, int s_want, int kvh) {
-    int first = 0;
-    for (int s = 0; s < s_want; ++s) first += ((dec_blocks(cu, s) + chunk - 1) / chunk) * Hkv;
-    const int per = (dec_blocks(cu, s_want) + chunk - 1) / chunk;
-    return make_int2(first + kvh * per, per);
 }
 
 // One CTA: per sequence the number of key blocks, a common chunk length (blocks per item) so that about
@@ -140,6 +167,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     volatile uint32_t* abort_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 68);
     volatile int* item_gen = reinterpret_cast<volatile int*>(smem_gen + L::kBars + 72);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    pdl_launch_dependents();                 // the merge kernel may get onto the SMs while this one runs
 
     // rows of the Q tile that no load ever writes must not hold NaN patterns: clear the tile once
     for (int i = tid * 16; i < L::kTileBytes; i += kDecThreads * 16) *reinterpret_cast<uint4*>(smem_gen + L::kQ + i) = make_uint4(0, 0, 0, 0);
@@ -160,13 +188,15 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();                              // set-up done; from here on the kernel in front has completed
     const uint32_t tmem = *tmem_slot_gen;
     const uint32_t tS = tmem, tP = tmem, tO = tmem + 128;
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, kDecBN, false, false);
     constexpr uint32_t idesc_o = idesc_bf16_f32(128, D, false, true);
     const bool self_plan = (p.plan == nullptr);
-    const int chunk = self_plan ? self_plan_chunk(p.cu, p.S, p.Hkv, p.target) : 0;
-    const int n_items = self_plan ? self_plan_count(p.cu, p.S, p.Hkv, chunk) : *p.n_items;
+    __shared__ SelfPlan sp;
+    if (self_plan) self_plan_build(sp, p.cu, p.S, p.Hkv, p.target);
+    const int n_items = self_plan ? sp.n_items : *p.n_items;
     uint32_t blk0 = 0, items_done = 0;       // barrier phases run on across the items of this CTA
 
     for (;;) {
@@ -180,7 +210,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         }
         if (item >= n_items || *abort_gen) break;
         tc_fence_after();
-        const DecItem it = self_plan ? self_plan_item(p.cu, p.S, p.Hkv, chunk, item) : p.plan[item];
+        const DecItem it = self_plan ? self_plan_item(sp, p.S, p.Hkv, item) : p.plan[item];
         const int seq_a = p.cu[it.s], len = p.cu[it.s + 1] - seq_a;
         const int nblk = it.b1 - it.b0;
         const int last_blk = (len + kDecBN - 1) / kDecBN - 1;       // the block of the sequence with a ragged end
@@ -389,9 +419,13 @@ decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ 
     __shared__ float s_red[kMergeThreads / 32];
     __shared__ float s_acc[kMergeGroups][128];
     __shared__ float s_m, s_l;
+    pdl_launch_dependents();
+    pdl_wait();                              // started while the decode kernel drains: its partial results are complete from here on
     const int s = blockIdx.x / Hq, h = blockIdx.x % Hq;
     const int kvh = h / G, row = h % G, Hkv = Hq / G;
-    const int2 sg = seg ? seg[s * Hkv + kvh] : self_plan_segment(cu, S, Hkv, self_plan_chunk(cu, S, Hkv, target), s, kvh);
+    __shared__ SelfPlan sp;
+    if (!seg) self_plan_build(sp, cu, S, Hkv, target);
+    const int2 sg = seg ? seg[s * Hkv + kvh] : make_int2(sp.first[s] + kvh * sp.per[s], sp.per[s]);
     const int cnt = sg.y < kMergeMaxSplits ? sg.y : kMergeMaxSplits;
     const size_t stride = (size_t)kDecRows * (D + 2);
     const float* base = partial + ((size_t)sg.x * kDecRows + row) * (D + 2);
@@ -472,8 +506,7 @@ static int launch_decode(const CUtensorMap& mq, const CUtensorMap& mk, const CUt
         if (cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
         configured = true;
     }
-    decode_kernel<D><<<grid, kDecThreads, smem, st>>>(mq, mk, mv, p, box_heads);
-    return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+    return launch_pdl(decode_kernel<D>, grid, kDecThreads, (size_t)smem, st, mq, mk, mv, p, box_heads) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 
 }  // namespace dash
@@ -506,7 +539,7 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
     int* seq_first = (int*)((char*)seg + align_up((size_t)S * Hkv * sizeof(int2), 256));
     float* partial = (float*)((char*)seq_first + align_up((size_t)S * sizeof(int), 256));
     const bool self_plan = S <= kSelfPlanSeqs;
-    const int target = 4 * sm_count();
+    const int target = 4 * sm_count();        // items aimed at: four per SM (self-planning CTAs go down to one item each where that keeps them all busy)
     if (!self_plan) {
         decode_plan_kernel<<<1, 256, 0, st>>>(cu_seqlens, S, Hkv, target, plan, seg, (int*)(w + 4), (unsigned int*)w, max_items, seq_first);
         DASH_CUDA_TRY(cudaGetLastError());
@@ -531,8 +564,7 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
         rc = D == 128 ? launch_decode<128>(mq, mk, mv, p, box_heads, grid, st) : launch_decode<64>(mq, mk, mv, p, box_heads, grid, st);
         if (rc != DASH_OK) return rc;
     }
-    decode_merge_kernel<false><<<S * Hq, kMergeThreads, 0, st>>>(partial, self_plan ? nullptr : seg, cu_seqlens, S, target, Hq, G, D, scale_log2, scale, out,
-                                                                ldo, lse);
-    DASH_CUDA_TRY(cudaGetLastError());
+    DASH_CUDA_TRY(launch_pdl(decode_merge_kernel<false>, S * Hq, kMergeThreads, 0, st, (const float*)partial, (const int2*)(self_plan ? nullptr : seg),
+                             cu_seqlens, S, target, Hq, G, D, scale_log2, scale, out, ldo, lse));
     return DASH_OK;
 }
