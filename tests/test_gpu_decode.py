@@ -49,6 +49,11 @@ def test_decode_qwen_heads_long_cache_split_over_many_ctas():
     _decode_case([100000], 28, 4, 128, 3)
 
 
+def test_decode_few_long_sequences_one_item_per_cta():
+    # unequal long caches whose keys are cut into one item per CTA (the last chunk of every sequence and head is shorter)
+    _decode_case([40000, 30001, 20000, 9000], 28, 4, 128, 7, pad=3)
+
+
 def test_decode_large_batch_takes_the_planned_path():
     # more sequences than the CTAs plan for themselves: items come from the plan kernel, by ticket
     g = torch.Generator().manual_seed(6)
