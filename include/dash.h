@@ -187,6 +187,26 @@ int dash_varlen_attention(const void* Q, const void* K, const void* V, void* O, 
                           int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
                           void* ws, size_t ws_bytes, void* stream);
 
+/* The same attention with Q left where it is (Sec. 3.4: the active tokens are "gathered";
+ * here the gathering happens inside the tile loads).  Q [n_full,Hq,D] is a full-length
+ * tensor; packed row i of the active set is its row idx[i] (device int32 [n], e.g.
+ * dash_compact's idx_out: ascending within a sequence).  kv_packed = 1: K, V [n,Hkv,D] are
+ * packed (compacted by the caller: 2 * 2 Hkv * D * es bytes per active token instead of
+ * 2 * (Hq + 2 Hkv) * D * es) -- the fast arrangement, a query tile is fetched once.
+ * kv_packed = 0: K, V [n_full,Hkv,D] are full-length too and every key block is fetched by
+ * index: no copy at all, but each query tile gathers its keys again, four rows per load --
+ * measured 2.5x slower than packed K, V (with packed K, V the call is within 1-3 % of
+ * dash_varlen_attention on packed Q).  cu_seqlens, S, n, max_seqlen describe the packed
+ * set as above; O [n,Hq,D] and lse [Hq,n] are written packed.  DASH_BF16 only
+ * (DASH_ERR_UNSUPPORTED for fp32); every idx[i] must lie in [0, n_full) -- not checked on
+ * the device. */
+int dash_varlen_attention_indexed(const void* Q, const void* K, const void* V, void* O, float* lse,
+                                  int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                                  const int32_t* idx, int64_t n_full, int kv_packed,
+                                  const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen,
+                                  int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
+                                  void* ws, size_t ws_bytes, void* stream);
+
 /* ---- decoding stage: one new token per sequence over the packed KV cache ---
  * (Preliminaries: decoding reuses the cached keys and values; Appendix C, "DASH settings":
  * halting prompt tokens shortens the KV cache -- the cache of a deeper layer holds only the

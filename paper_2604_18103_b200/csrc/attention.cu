@@ -49,6 +49,20 @@ int make_map_rows_heads(CUtensorMap* map, const void* base, int64_t rows, int he
     return r == CUDA_SUCCESS ? DASH_OK : DASH_ERR_CUDA;
 }
 
+// bf16 tensor [rows, cols] (cols = heads * D), box = 64 columns of one row: the map of the four-row gather loads
+int make_map_rows_gather(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return DASH_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, 1};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DASH_OK : DASH_ERR_CUDA;
+}
+
 constexpr int kBM = 128;                 // query rows per CTA
 constexpr int kBN = 128;                 // keys per block
 constexpr int kAttnThreads = 160;
@@ -73,6 +87,8 @@ struct AttnParams {
     const int2* plan;           // (sequence, query tile) of every item group, heaviest first; Hq items (heads) per entry
     const int* n_items;         // device: entries * Hq
     unsigned int* ticket;       // device: next item to hand out
+    const int32_t* idx;         // GATHER: packed row i is row idx[i] of the full-length Q (and of K, V unless kv_packed)
+    int kv_packed;              // GATHER: K and V are packed already ([n, Hkv, D], tiled loads); only Q is fetched by index
 };
 
 // ---- plan: which (sequence, query tile) pairs exist, ordered by falling number of key blocks ----
@@ -133,7 +149,10 @@ struct AttnSmem {
     static constexpr int kTotal = kBars + 128;
 };
 
-template <int D, bool OUT_F32>
+// GATHER: Q, K and V are full-length [rows, heads * D] tensors and the packed active set is given by p.idx; tiles are fetched four
+// rows per instruction (TMA gather4, issued by all lanes of warp 4: lane l brings rows 4l .. 4l+3 of the tile), so the active rows
+// of Q, K, V are never copied into packed buffers.  Everything else -- and the packed O -- is the same.
+template <int D, bool OUT_F32, bool GATHER>
 __global__ void __launch_bounds__(kAttnThreads, 2)
 attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                  const __grid_constant__ CUtensorMap mapV, const AttnParams p) {
@@ -197,11 +216,83 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const int nblk = qt + 1;                                 // causal: key blocks 0..qt
     const uint32_t qph = items_done & 1;
 
-    if (warp == 4) {
+    // tile of 128 packed rows starting at row0, fetched by index: lane l of warp 4 brings rows 4l .. 4l+3
+    auto gather_tile = [&](uint32_t sT, const CUtensorMap* map, uint32_t bar, int head, int row0) {
+        if (GATHER) {
+            if (lane == 0) mbar_arrive_expect_tx(bar, L::kTileBytes);
+            __syncwarp();
+            int r[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int pr = row0 + 4 * lane + k;                  // rows past the sequence's end: its last row again (masked / zeroed later)
+                r[k] = p.idx[pr < seq_b ? pr : seq_b - 1];
+            }
+#pragma unroll
+            for (int c = 0; c < KCH; ++c) tma_gather4(sT + c * kChunkBytes + lane * 512, map, bar, head * D + c * 64, r[0], r[1], r[2], r[3]);
+        }
+    };
+    if (warp == 4 && GATHER && !p.kv_packed) {
+        // K and V by index as well: the schedule of the branch below with the whole warp in step -- lane 0 issues the MMAs, every
+        // lane its share of the loads (the waits of 32 lanes and their votes cost about 500 cycles per key block)
+        bool ok = true;
+        auto all_ok = [&](bool v) { return __all_sync(0xffffffffu, v) != 0; };
+        auto issue_s = [&]() {
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = (kk >> 2) * kChunkBytes + (kk & 3) * 32;
+                mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), idesc_s, kk > 0);
+            }
+            tc_commit(bar_s);
+        };
+        auto load_kv = [&](uint32_t sT, const CUtensorMap* map, uint32_t bar, int row0) { gather_tile(sT, map, bar, kvh, row0); };
+        gather_tile(sQ, &mapQ, bar_q, h, seq_a + q0);
+        load_kv(sK, &mapK, bar_k, seq_a);
+        load_kv(sV, &mapV, bar_v, seq_a);
+        ok = all_ok(mbar_wait(bar_q, qph, kWaitCycles) && mbar_wait(bar_k, blk0 & 1, kWaitCycles));
+        if (ok && lane == 0) issue_s();
+        __syncwarp();
+        for (int j = 0; j < nblk && ok; ++j) {
+            const uint32_t ph = (blk0 + j) & 1;
+            ok = all_ok(mbar_wait(bar_s, ph, kWaitCycles));                   // S_j done: the K buffer is free
+            if (!ok) break;
+            if (j + 1 < nblk) load_kv(sK, &mapK, bar_k, seq_a + (j + 1) * kBN);
+            ok = all_ok(mbar_wait(bar_p0, ph, kWaitCycles) && mbar_wait(bar_v, ph, kWaitCycles));
+            if (!ok) break;
+            if (lane == 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < kBN / 32; ++kk)
+                    mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
+            }
+            ok = all_ok(mbar_wait(bar_p1, ph, kWaitCycles));
+            if (!ok) break;
+            if (lane == 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int kk = kBN / 32; kk < kBN / 16; ++kk)
+                    mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, 1);
+                tc_commit(bar_o);
+            }
+            if (j + 1 < nblk) {
+                ok = all_ok(mbar_wait(bar_k, (blk0 + j + 1) & 1, kWaitCycles));
+                if (!ok) break;
+                if (lane == 0) issue_s();
+            }
+            ok = all_ok(mbar_wait(bar_o, ph, kWaitCycles));                   // PV_j done: the V buffer is free
+            if (!ok) break;
+            if (j + 1 < nblk) load_kv(sV, &mapV, bar_v, seq_a + (j + 1) * kBN);
+        }
+        if (!ok && lane == 0) { *abort_gen = 1; atomicExch(p.status, DASH_ERR_TIMEOUT); }
+    } else if (warp == 4) {
+        // Q by index (K and V packed): the whole warp fetches the query tile, then lane 0 runs the item as for packed tensors
+        if (GATHER) gather_tile(sQ, &mapQ, bar_q, h, seq_a + q0);
         if (lane == 0) {
             bool ok = true;
-            mbar_arrive_expect_tx(bar_q, L::kTileBytes);
-            for (int c = 0; c < KCH; ++c) tma_load_3d(sQ + c * kChunkBytes, &mapQ, bar_q, c * 64, h, seq_a + q0);
+            if (!GATHER) {
+                mbar_arrive_expect_tx(bar_q, L::kTileBytes);
+                for (int c = 0; c < KCH; ++c) tma_load_3d(sQ + c * kChunkBytes, &mapQ, bar_q, c * 64, h, seq_a + q0);
+            }
             mbar_arrive_expect_tx(bar_k, L::kTileBytes);
             for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, kvh, seq_a);
             mbar_arrive_expect_tx(bar_v, L::kTileBytes);
@@ -435,16 +526,16 @@ size_t attention_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D, dash_dtype d
     return b;
 }
 
-template <int D, bool OUT_F32>
+template <int D, bool OUT_F32, bool GATHER>
 static int launch_attention(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p, int grid, cudaStream_t st) {
     using L = AttnSmem<D>;
     const int smem = L::kTotal + 1024;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(attention_kernel<D, OUT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
+        if (cudaFuncSetAttribute(attention_kernel<D, OUT_F32, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
         configured = true;
     }
-    return launch_pdl(attention_kernel<D, OUT_F32>, grid, kAttnThreads, (size_t)smem, st, mq, mk, mv, p) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+    return launch_pdl(attention_kernel<D, OUT_F32, GATHER>, grid, kAttnThreads, (size_t)smem, st, mq, mk, mv, p) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 
 // The item list of a call (see attention_plan_kernel) into the head of its workspace.  A caller that knows cu_seqlens early
@@ -463,7 +554,8 @@ static int attention_impl(const void* Q, const void* K, const void* V, void* O, 
                           int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
                           const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen,
                           int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
-                          void* ws, size_t ws_bytes, void* stream, bool planned) {
+                          void* ws, size_t ws_bytes, void* stream, bool planned, const int32_t* idx = nullptr, int64_t n_full = 0,
+                          bool kv_packed = false) {
     if (n < 0 || S < 1 || max_seqlen < 0 || Hq < 1 || Hkv < 1 || !cu_seqlens) return DASH_ERR_INVALID_ARG;
     if (dt != DASH_F32 && dt != DASH_BF16) return DASH_ERR_INVALID_ARG;
     if (D != 64 && D != 128) return DASH_ERR_UNSUPPORTED;
@@ -482,6 +574,7 @@ static int attention_impl(const void* Q, const void* K, const void* V, void* O, 
     const void *q = Q, *k = K, *v = V;
     int64_t lq = ldq, lk = ldk, lv = ldv;
     if (!ws || ((uintptr_t)ws % 256) || ws_bytes < attention_ws_bytes(n, S, Hq, Hkv, D, dt)) return DASH_ERR_WORKSPACE;
+    if (idx && (dt != DASH_BF16 || n_full < 1 || n_full > 0x7fffffffLL)) return dt != DASH_BF16 ? DASH_ERR_UNSUPPORTED : DASH_ERR_INVALID_ARG;
     if (dt == DASH_F32) {
         __nv_bfloat16* qb = (__nv_bfloat16*)((char*)ws + 256 + plan_bytes(n, S));
         __nv_bfloat16* kb = qb + (size_t)n * Hq * D;
@@ -500,16 +593,27 @@ static int attention_impl(const void* Q, const void* K, const void* V, void* O, 
     }
     CUtensorMap mq, mk, mv;
     int rc;
-    if ((rc = make_map_rows_heads(&mq, q, n, Hq, D, lq, kBM)) != DASH_OK) return rc;
-    if ((rc = make_map_rows_heads(&mk, k, n, Hkv, D, lk, kBN)) != DASH_OK) return rc;
-    if ((rc = make_map_rows_heads(&mv, v, n, Hkv, D, lv, kBN)) != DASH_OK) return rc;
+    if (idx) {
+        if ((rc = make_map_rows_gather(&mq, q, n_full, (int64_t)Hq * D, lq)) != DASH_OK) return rc;
+        if (kv_packed) {
+            if ((rc = make_map_rows_heads(&mk, k, n, Hkv, D, lk, kBN)) != DASH_OK) return rc;
+            if ((rc = make_map_rows_heads(&mv, v, n, Hkv, D, lv, kBN)) != DASH_OK) return rc;
+        } else {
+            if ((rc = make_map_rows_gather(&mk, k, n_full, (int64_t)Hkv * D, lk)) != DASH_OK) return rc;
+            if ((rc = make_map_rows_gather(&mv, v, n_full, (int64_t)Hkv * D, lv)) != DASH_OK) return rc;
+        }
+    } else {
+        if ((rc = make_map_rows_heads(&mq, q, n, Hq, D, lq, kBM)) != DASH_OK) return rc;
+        if ((rc = make_map_rows_heads(&mk, k, n, Hkv, D, lk, kBN)) != DASH_OK) return rc;
+        if ((rc = make_map_rows_heads(&mv, v, n, Hkv, D, lv, kBN)) != DASH_OK) return rc;
+    }
 
     AttnParams p;
     p.cu = cu_seqlens; p.S = S; p.Hq = Hq; p.Hkv = Hkv;
     p.n_qtiles = (int)((max_seqlen + kBM - 1) / kBM);
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.O = O; p.ldo = ldo; p.lse = lse; p.n = n;
+    p.O = O; p.ldo = ldo; p.lse = lse; p.n = n; p.idx = idx; p.kv_packed = kv_packed ? 1 : 0;
     p.status = status_word_ptr();
     if (!p.status) return DASH_ERR_CUDA;
     p.ticket = (unsigned int*)ws;
@@ -520,8 +624,9 @@ static int attention_impl(const void* Q, const void* K, const void* V, void* O, 
     int64_t grid64 = (int64_t)p.n_qtiles * Hq * S;
     if (grid64 > 2LL * sm_count()) grid64 = 2LL * sm_count();
     const int grid = (int)grid64;
-    if (D == 128) return dt == DASH_F32 ? launch_attention<128, true>(mq, mk, mv, p, grid, st) : launch_attention<128, false>(mq, mk, mv, p, grid, st);
-    return dt == DASH_F32 ? launch_attention<64, true>(mq, mk, mv, p, grid, st) : launch_attention<64, false>(mq, mk, mv, p, grid, st);
+    if (idx) return D == 128 ? launch_attention<128, false, true>(mq, mk, mv, p, grid, st) : launch_attention<64, false, true>(mq, mk, mv, p, grid, st);
+    if (D == 128) return dt == DASH_F32 ? launch_attention<128, true, false>(mq, mk, mv, p, grid, st) : launch_attention<128, false, false>(mq, mk, mv, p, grid, st);
+    return dt == DASH_F32 ? launch_attention<64, true, false>(mq, mk, mv, p, grid, st) : launch_attention<64, false, false>(mq, mk, mv, p, grid, st);
 }
 
 // same as dash_varlen_attention for a workspace whose item list attention_plan() has already been asked for on this stream
@@ -540,4 +645,16 @@ extern "C" int dash_varlen_attention(const void* Q, const void* K, const void* V
                                      void* ws, size_t ws_bytes, void* stream) {
     return dash::attention_impl(Q, K, V, O, lse, ldq, ldk, ldv, ldo, cu_seqlens, S, n, max_seqlen, Hq, Hkv, D, scale, causal, dt, ws, ws_bytes,
                                 stream, false);
+}
+
+extern "C" int dash_varlen_attention_indexed(const void* Q, const void* K, const void* V, void* O, float* lse,
+                                             int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
+                                             const int32_t* idx, int64_t n_full, int kv_packed,
+                                             const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen,
+                                             int Hq, int Hkv, int D, float scale, int causal, dash_dtype dt,
+                                             void* ws, size_t ws_bytes, void* stream) {
+    if ((!idx && n > 0) || (kv_packed != 0 && kv_packed != 1)) return DASH_ERR_INVALID_ARG;
+    if (n > n_full) return DASH_ERR_INVALID_ARG;
+    return dash::attention_impl(Q, K, V, O, lse, ldq, ldk, ldv, ldo, cu_seqlens, S, n, max_seqlen, Hq, Hkv, D, scale, causal, dt, ws, ws_bytes,
+                                stream, false, idx, n_full, kv_packed != 0);
 }

@@ -29,7 +29,7 @@ EXPORTS = [
     "dash_status_string", "dash_check_status", "dash_keep_count", "dash_flops_per_layer", "dash_flops_speedup",
     "dash_delta_norm", "dash_select", "dash_compact", "dash_scatter", "dash_varlen_attention",
     "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes", "dash_compact_static",
-    "dash_block_workspace", "dash_block_step", "dash_decode_attention",
+    "dash_block_workspace", "dash_block_step", "dash_decode_attention", "dash_varlen_attention_indexed",
 ]
 COMPACT_STATIC_MAX_ROWS = 1 << 20
 
@@ -98,6 +98,9 @@ def lib() -> ctypes.CDLL:
         L.dash_varlen_attention.argtypes = [c_void_p] * 5 + [c_int64] * 4 + [c_void_p, c_int, c_int64, c_int64,
                                                                           c_int, c_int, c_int, c_float, c_int, c_int,
                                                                           c_void_p, c_size_t, c_void_p]
+        L.dash_varlen_attention_indexed.argtypes = [c_void_p] * 5 + [c_int64] * 4 + [c_void_p, c_int64, c_int, c_void_p, c_int, c_int64, c_int64,
+                                                                                  c_int, c_int, c_int, c_float, c_int, c_int,
+                                                                                  c_void_p, c_size_t, c_void_p]
         L.dash_layer_workspace.argtypes = [POINTER(LayerCfg), c_int64, c_int, POINTER(LayerWsLayout)]
         L.dash_layer_step.argtypes = [POINTER(LayerCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -278,6 +281,34 @@ def dash_varlen_attention(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, cu_
                                      _p(cu_seqlens), cu_seqlens.numel() - 1, n, int(max_seqlen), Hq, Hkv, D, float(scale), 1, dt,
                                      _p(ws), ws.numel(), _stream())
     _check(st, "dash_varlen_attention")
+    return (O, lse) if want_lse else O
+
+
+def dash_varlen_attention_indexed(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, idx: torch.Tensor, cu_seqlens: torch.Tensor,
+                                  max_seqlen: int, n: Optional[int] = None, kv_packed: bool = False, scale: Optional[float] = None,
+                                  O: Optional[torch.Tensor] = None, want_lse: bool = False, ws: Optional[torch.Tensor] = None):
+    """Q [n_full,Hq,D] full-length (bf16); packed row i of the active set is its row idx[i].  K, V: packed [n,Hkv,D]
+    (kv_packed=True, the fast arrangement) or full-length [n_full,Hkv,D] fetched by idx as well.
+    n: rows of the packed set allocated (default: idx.numel()).  Returns the packed O [n,Hq,D] (and lse [Hq,n] if asked)."""
+    _dev(Q, K, V, idx, cu_seqlens)
+    n_full, Hq, D = Q.shape
+    Hkv = K.shape[1]
+    if n is None:
+        n = idx.numel()
+    if idx.dtype != torch.int32 or idx.numel() < n:
+        raise ValueError("idx must be int32 with at least n entries")
+    if scale is None:
+        scale = 1.0 / (D ** 0.5)
+    if O is None:
+        O = torch.empty(n, Hq, D, dtype=Q.dtype, device=Q.device)
+    lse = torch.empty(Hq, n, dtype=torch.float32, device=Q.device) if want_lse else None
+    dt = dtype_code(Q)
+    if ws is None:
+        ws = workspace(dash_workspace_bytes(WS_ATTENTION, n, cu_seqlens.numel() - 1, Hq, Hkv, D, dt), Q.device)
+    st = lib().dash_varlen_attention_indexed(_p(Q), _p(K), _p(V), _p(O), _p(lse), Q.stride(0), K.stride(0), V.stride(0), O.stride(0),
+                                             _p(idx), n_full, int(bool(kv_packed)), _p(cu_seqlens), cu_seqlens.numel() - 1, n, int(max_seqlen), Hq, Hkv, D,
+                                             float(scale), 1, dt, _p(ws), ws.numel(), _stream())
+    _check(st, "dash_varlen_attention_indexed")
     return (O, lse) if want_lse else O
 
 

@@ -203,6 +203,50 @@ def _attention_case(lengths, Hq, Hkv, D, dtype, seed, rows=None, pad=0, tol=TOL)
     assert np.allclose(got_lse, lref, atol=2e-2), float(np.max(np.abs(got_lse - lref)))
 
 
+def _indexed_attention_case(full_lengths, keep_prob, Hq, Hkv, D, seed, tol=TOL):
+    """Full-length Q, K, V with a random subset of every sequence active; the rows that are not active hold NaN / Inf, so any
+    read of them would show.  The index-driven kernel must equal the oracle's attention over the gathered rows."""
+    g = torch.Generator().manual_seed(seed)
+    cu_full = wl.cu_from_lengths(full_lengths)
+    n_full = int(cu_full[-1])
+    mask = torch.rand(n_full, generator=g) < keep_prob
+    idx = torch.nonzero(mask).flatten().to(torch.int32)
+    lengths = [int(mask[int(cu_full[s]):int(cu_full[s + 1])].sum()) for s in range(len(full_lengths))]
+    cu = wl.cu_from_lengths(lengths)
+    n = int(cu[-1])
+    Q = torch.randn(n_full, Hq, D, generator=g).to(torch.bfloat16)
+    K = torch.randn(n_full, Hkv, D, generator=g).to(torch.bfloat16)
+    V = torch.randn(n_full, Hkv, D, generator=g).to(torch.bfloat16)
+    Qp, Kp, Vp = Q.clone(), K.clone(), V.clone()
+    Qp[~mask], Kp[~mask], Vp[~mask] = float("nan"), float("inf"), float("nan")
+    O, lse = dash.dash_varlen_attention_indexed(Qp.to(DEV), Kp.to(DEV), Vp.to(DEV), idx.to(DEV), cu.to(DEV), max(max(lengths), 1), want_lse=True)
+    torch.cuda.synchronize()
+    assert dash.dash_check_status() == dash.OK
+    sel = idx.long()
+    Oref, lref = oc.attention(Q[sel], K[sel], V[sel], cu)
+    assert_close_rms(O.float().cpu().numpy(), Oref, f"indexed O {full_lengths} keep {keep_prob} Hq{Hq} D{D}", tol=tol)
+    assert np.allclose(lse.cpu().numpy().T, lref, atol=2e-2)
+    # the same numbers as the kernel on packed copies of the active rows (same arithmetic, other loads)
+    Kc, Vc = K[sel].contiguous().to(DEV), V[sel].contiguous().to(DEV)
+    O2 = dash.dash_varlen_attention(Q[sel].contiguous().to(DEV), Kc, Vc, cu.to(DEV), max(max(lengths), 1))
+    assert torch.equal(O.cpu(), O2.cpu())
+    # Q by index, K and V packed by the caller
+    O3 = dash.dash_varlen_attention_indexed(Qp.to(DEV), Kc, Vc, idx.to(DEV), cu.to(DEV), max(max(lengths), 1), kv_packed=True)
+    assert torch.equal(O.cpu(), O3.cpu())
+
+
+def test_indexed_attention_ragged_tiles_gqa():
+    _indexed_attention_case([700], 0.45, 4, 2, 128, 21)
+
+
+def test_indexed_attention_packed_batch_with_an_empty_active_set():
+    _indexed_attention_case([400, 130, 3, 900], 0.3, 14, 2, 128, 22)
+
+
+def test_indexed_attention_head_dim_64_and_keep_all():
+    _indexed_attention_case([517], 1.1, 4, 4, 64, 23)
+
+
 def test_attention_single_tile():
     _attention_case([128], 1, 1, 128, torch.bfloat16, 1)
 
