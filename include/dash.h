@@ -73,6 +73,16 @@ int dash_check_status(void* stream);
  * stay and floor(round(rho * (n - keep_first - keep_last))) of the others are
  * dropped (round = to nearest, ties to even).  Returns -1 on invalid input. */
 int64_t dash_keep_count(int64_t n, double rho, int keep_first, int keep_last, int mode);
+
+/* The same kept lengths on the device, one per sequence, from the sequence lengths as they
+ * stand in cu_seqlens (device int32 [S+1]): keep_counts_out[s] (device int32 [S]) =
+ * dash_keep_count(cu[s+1] - cu[s], ...), the same fp64 arithmetic.  For dash_select's
+ * keep-count rule in layers whose entering lengths exist only on the device (behind a
+ * selecting layer), so that no length has to come back to the host.  Asynchronous on
+ * `stream`.  DASH_ERR_INVALID_ARG for null pointers, S < 1, rho outside [0, 1), negative
+ * keep_first / keep_last or a mode other than 0 / 1. */
+int dash_keep_counts_device(const int32_t* cu_seqlens, int S, double rho, int keep_first, int keep_last,
+                            int mode, int32_t* keep_counts_out, void* stream);
 /* Appendix A FLOPs proxy of one block: A(n) = 4 n d^2 + 2 n^2 d + 2 n d m. */
 double dash_flops_per_layer(double n, double d, double m);
 /* Appendix A: C_full / C_ours with C_full = L A(n), C_ours = l_s A(n) + (L - l_s) A(n_hat). */

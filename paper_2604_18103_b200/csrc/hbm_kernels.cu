@@ -669,6 +669,31 @@ extern "C" int dash_select(const float* r, int64_t n, const int32_t* cu_seqlens,
     return DASH_OK;
 }
 
+// keep_counts[s] from the length of sequence s as it stands on the device: the arithmetic of dash_keep_count, in fp64
+__global__ void __launch_bounds__(256)
+keep_counts_kernel(const int32_t* __restrict__ cu, int S, double rho, int keep_first, int keep_last, int mode, int32_t* __restrict__ out) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= S) return;
+    const long long n = (long long)cu[s + 1] - cu[s];
+    long long k;
+    if (mode == 0) {
+        k = (long long)floor(__dmul_rn(__dsub_rn(1.0, rho), (double)n));
+    } else {
+        long long n_fix = (long long)keep_first + keep_last;
+        if (n_fix > n) n_fix = n;
+        k = n - (long long)floor(rint(__dmul_rn(rho, (double)(n - n_fix))));      // rint: to nearest, ties to even
+    }
+    out[s] = (int32_t)(k < 0 ? 0 : (k > n ? n : k));
+}
+
+extern "C" int dash_keep_counts_device(const int32_t* cu_seqlens, int S, double rho, int keep_first, int keep_last, int mode,
+                                       int32_t* keep_counts_out, void* stream) {
+    if (!cu_seqlens || !keep_counts_out || S < 1 || !(rho >= 0.0) || !(rho < 1.0) || keep_first < 0 || keep_last < 0 || (mode != 0 && mode != 1))
+        return DASH_ERR_INVALID_ARG;
+    keep_counts_kernel<<<(S + 255) / 256, 256, 0, (cudaStream_t)stream>>>(cu_seqlens, S, rho, keep_first, keep_last, mode, keep_counts_out);
+    return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+}
+
 // Tokens per CTA.  Small tiles keep the CTAs balanced when the active rows cluster (a packed batch whose
 // image blocks halt almost entirely while its text blocks stay); larger ones only bound the look-back chain.
 static int compact_tile_for(int64_t n) {

@@ -30,6 +30,7 @@ EXPORTS = [
     "dash_delta_norm", "dash_select", "dash_compact", "dash_scatter", "dash_varlen_attention",
     "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes", "dash_compact_static",
     "dash_block_workspace", "dash_block_step", "dash_decode_attention", "dash_varlen_attention_indexed",
+    "dash_keep_counts_device",
 ]
 COMPACT_STATIC_MAX_ROWS = 1 << 20
 
@@ -101,6 +102,7 @@ def lib() -> ctypes.CDLL:
         L.dash_varlen_attention_indexed.argtypes = [c_void_p] * 5 + [c_int64] * 4 + [c_void_p, c_int64, c_int, c_void_p, c_int, c_int64, c_int64,
                                                                                   c_int, c_int, c_int, c_float, c_int, c_int,
                                                                                   c_void_p, c_size_t, c_void_p]
+        L.dash_keep_counts_device.argtypes = [c_void_p, c_int, c_double, c_int, c_int, c_int, c_void_p, c_void_p]
         L.dash_layer_workspace.argtypes = [POINTER(LayerCfg), c_int64, c_int, POINTER(LayerWsLayout)]
         L.dash_layer_step.argtypes = [POINTER(LayerCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -208,6 +210,18 @@ def dash_select(r: torch.Tensor, cu_seqlens: torch.Tensor, mode: int, tau: float
                            _p(mask_out), None, 0, _stream())
     _check(st, "dash_select")
     return mask_out
+
+
+def dash_keep_counts_device(cu_seqlens: torch.Tensor, rho: float, keep_first: int = 0, keep_last: int = 0, mode: int = 0,
+                            out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Kept length of every sequence (int32 [S], on the device) from the lengths in cu_seqlens: no host round trip."""
+    _dev(cu_seqlens)
+    S = cu_seqlens.numel() - 1
+    if out is None:
+        out = torch.empty(S, dtype=torch.int32, device=cu_seqlens.device)
+    st = lib().dash_keep_counts_device(_p(cu_seqlens), S, float(rho), keep_first, keep_last, mode, _p(out), _stream())
+    _check(st, "dash_keep_counts_device")
+    return out
 
 
 # ---- step 3 ---------------------------------------------------------------------

@@ -118,6 +118,25 @@ def test_select_matches_oracle(lengths):
             assert np.array_equal(m.cpu().numpy(), ref), (lengths, kf, kl, frac)
 
 
+def test_keep_counts_on_the_device_equal_the_oracle_and_feed_the_keep_count_rule():
+    """Kept lengths computed on the device from cu_seqlens (Eq. 3 and the Appendix-A rule): bit-equal to the oracle's for the
+    paper's prompt lengths, for random lengths and for the degenerate ones; then used by the keep-count rule without a host copy."""
+    g = torch.Generator().manual_seed(77)
+    lengths = [8192, 16384, 32768, 65536, 131072, 0, 1, 95, 96, 97] + torch.randint(0, 200000, (300,), generator=g).tolist()
+    cu = wl.cu_from_lengths(lengths).to(DEV)
+    for rho, kf, kl, mode in ((0.4, 0, 0, 0), (0.667, 64, 32, 1), (0.5, 64, 32, 1), (0.0, 0, 0, 0), (0.999, 3, 5, 1), (0.8, 0, 0, 0)):
+        got = dash.dash_keep_counts_device(cu, rho, kf, kl, mode).cpu().tolist()
+        assert got == [oc.keep_count(L, rho, kf, kl, mode) for L in lengths], (rho, kf, kl, mode)
+    lengths = [5000, 300, 0, 1700]
+    cu_h = wl.cu_from_lengths(lengths)
+    n = int(cu_h[-1])
+    r = torch.exp(torch.randn(n, generator=g) - 3.0)
+    Kd = dash.dash_keep_counts_device(cu_h.to(DEV), 0.667, 64, 32, 1)
+    m = dash.dash_select(r.to(DEV), cu_h.to(DEV), dash.SEL_KEEP_COUNT, keep_counts=Kd, keep_first=64, keep_last=32)
+    Ks = [oc.keep_count(L, 0.667, 64, 32, 1) for L in lengths]
+    assert np.array_equal(m.cpu().numpy(), oc.select(r.numpy(), cu_h, oc.KEEP_COUNT, keep_counts=Ks, keep_first=64, keep_last=32))
+
+
 def test_select_high_direction_matches_oracle():
     lengths = [300, 0, 1700, 1]
     cu = wl.cu_from_lengths(lengths)
