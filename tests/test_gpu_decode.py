@@ -63,6 +63,25 @@ def test_decode_large_batch_takes_the_planned_path():
     _decode_case(lengths, 14, 2, 128, 6, pad=7)
 
 
+def test_decode_random_batches_match_oracle():
+    """Seeded sweep over batch sizes on both sides of the self-planning limit, length mixes (many short, one long, equal,
+    block-aligned), head groupings and head dims."""
+    g = torch.Generator().manual_seed(2024)
+    for trial in range(16):
+        S = int(torch.randint(1, 41, (1,), generator=g))
+        kind = trial % 4
+        if kind == 0:
+            lens = torch.randint(0, 3000, (S,), generator=g).tolist()
+        elif kind == 1:
+            lens = [int(torch.randint(1, 60000, (1,), generator=g))] + torch.randint(0, 300, (S - 1,), generator=g).tolist()
+        elif kind == 2:
+            lens = [int(torch.randint(100, 9000, (1,), generator=g))] * S
+        else:
+            lens = (torch.randint(0, 40, (S,), generator=g) * 128).tolist()
+        Hkv, G, D = [1, 2, 4][trial % 3], [1, 4, 7, 8][trial % 4], [64, 128][trial % 2]
+        _decode_case(lens, Hkv * G, Hkv, D, 100 + trial)
+
+
 def test_decode_head_dim_64_no_grouping_and_wide_grouping():
     _decode_case([777, 2000], 4, 4, 64, 4)
     _decode_case([1500], 8, 1, 64, 5, pad=3)

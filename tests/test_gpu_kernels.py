@@ -266,6 +266,41 @@ def test_indexed_attention_head_dim_64_and_keep_all():
     _indexed_attention_case([517], 1.1, 4, 4, 64, 23)
 
 
+def test_indexed_attention_random_shapes_equal_the_packed_kernel():
+    """Seeded sweep: sequence counts, lengths (also multiples of the tile), keep fractions from 5 % to all, head groupings,
+    head dims; the index-driven kernel (both arrangements of K, V) must reproduce the packed kernel bit for bit."""
+    g = torch.Generator().manual_seed(2025)
+    for trial in range(12):
+        S = int(torch.randint(1, 6, (1,), generator=g))
+        full = torch.randint(1, 1500, (S,), generator=g).tolist()
+        if trial % 5 == 0:
+            full = [128 * int(torch.randint(1, 8, (1,), generator=g)) for _ in range(S)]
+        keep = [0.05, 0.3, 0.7, 1.1][trial % 4]
+        Hkv, G, D = [1, 2, 4][trial % 3], [1, 2, 7][trial % 3], [128, 64][trial % 2]
+        Hq = Hkv * G
+        cu_full = wl.cu_from_lengths(full)
+        n_full = int(cu_full[-1])
+        mask = torch.rand(n_full, generator=g) < keep
+        idx = torch.nonzero(mask).flatten().to(torch.int32)
+        lens = [int(mask[int(cu_full[s]):int(cu_full[s + 1])].sum()) for s in range(S)]
+        cu = wl.cu_from_lengths(lens)
+        if int(cu[-1]) == 0:
+            continue
+        Q = torch.randn(n_full, Hq, D, generator=g).to(torch.bfloat16)
+        K = torch.randn(n_full, Hkv, D, generator=g).to(torch.bfloat16)
+        V = torch.randn(n_full, Hkv, D, generator=g).to(torch.bfloat16)
+        Qp, Kp, Vp = Q.clone(), K.clone(), V.clone()
+        Qp[~mask], Kp[~mask], Vp[~mask] = float("nan"), float("inf"), float("nan")
+        sel, ms = idx.long(), max(max(lens), 1)
+        Kc, Vc = K[sel].contiguous().to(DEV), V[sel].contiguous().to(DEV)
+        O1 = dash.dash_varlen_attention(Q[sel].contiguous().to(DEV), Kc, Vc, cu.to(DEV), ms)
+        O2 = dash.dash_varlen_attention_indexed(Qp.to(DEV), Kp.to(DEV), Vp.to(DEV), idx.to(DEV), cu.to(DEV), ms)
+        O3 = dash.dash_varlen_attention_indexed(Qp.to(DEV), Kc, Vc, idx.to(DEV), cu.to(DEV), ms, kv_packed=True)
+        torch.cuda.synchronize()
+        assert dash.dash_check_status() == dash.OK
+        assert torch.isfinite(O1.float()).all() and torch.equal(O1, O2) and torch.equal(O1, O3), (trial, full, keep)
+
+
 def test_attention_single_tile():
     _attention_case([128], 1, 1, 128, torch.bfloat16, 1)
 
