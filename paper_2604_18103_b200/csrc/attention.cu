@@ -14,6 +14,10 @@
 //   exp2, row sum, P (bf16) back into TMEM, rescale O if the max moved  ->
 //   O += P V_j  (TS MMA: A operand read from TMEM)
 // Causal tile skipping: a query tile only visits key blocks 0..its own index.
+//
+// The kernel is launched to start while the kernel in front of it in the stream drains (barriers, TMEM and descriptor prefetch are
+// set up before griddepcontrol.wait).  A second instantiation (GATHER) takes the query rows -- and, optionally, the key / value
+// rows -- of the packed set by index from full-length tensors (TMA gather4 loads) instead of from packed copies.
 #include <math.h>
 
 #include "common.cuh"
