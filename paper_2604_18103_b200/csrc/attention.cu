@@ -88,7 +88,7 @@ struct AttnParams {
     float* lse;             // [Hq, n] or null
     int64_t n;
     int* status;
-    const int2* plan;           // (sequence, query tile) of every item group, heaviest first; Hq items (heads) per entry
+    const int4* plan;           // (sequence, query tile, first row, end row of the sequence) of every item group, heaviest first; Hq items (heads) per entry
     const int* n_items;         // device: entries * Hq
     unsigned int* ticket;       // device: next item to hand out
     const int32_t* idx;         // GATHER: packed row i is row idx[i] of the full-length Q (and of K, V unless kv_packed)
@@ -97,7 +97,7 @@ struct AttnParams {
 
 // ---- plan: which (sequence, query tile) pairs exist, ordered by falling number of key blocks ----
 __global__ void __launch_bounds__(1024)
-attention_plan_kernel(const int32_t* __restrict__ cu, int S, int Hq, int2* __restrict__ plan, int* __restrict__ n_items,
+attention_plan_kernel(const int32_t* __restrict__ cu, int S, int Hq, int4* __restrict__ plan, int* __restrict__ n_items,
                       unsigned int* __restrict__ ticket, int64_t max_entries) {
     __shared__ int s_warp[33];
     __shared__ int s_max;
@@ -135,7 +135,7 @@ attention_plan_kernel(const int32_t* __restrict__ cu, int S, int Hq, int2* __res
         const int chunk_total = s_warp[32];
         if (qt >= 0)
             for (int s = 0; s < S; ++s)
-                if ((cu[s + 1] - cu[s] + kBM - 1) / kBM > qt) { if (k < max_entries) plan[k] = make_int2(s, qt); ++k; }
+                if ((cu[s + 1] - cu[s] + kBM - 1) / kBM > qt) { if (k < max_entries) plan[k] = make_int4(s, qt, cu[s], cu[s + 1]); ++k; }
         offset += chunk_total;
         __syncthreads();
     }
@@ -211,10 +211,10 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     if (item >= n_items || *abort_gen) break;
     tc_fence_after();
     // the heads of one KV group run next to each other, so their K/V tiles are shared through L2
-    const int2 e = p.plan[item / p.Hq];
-    const int h = item % p.Hq, s = e.x, qt = e.y;
+    const int4 e = p.plan[item / p.Hq];                      // one load: the sequence's bounds ride along with the entry
+    const int h = item % p.Hq, qt = e.y;
     const int kvh = h / G;
-    const int seq_a = p.cu[s], seq_b = p.cu[s + 1];
+    const int seq_a = e.z, seq_b = e.w;
     const int len = seq_b - seq_a;
     const int q0 = qt * kBM;
     const int nblk = qt + 1;                                 // causal: key blocks 0..qt
@@ -520,10 +520,10 @@ __global__ void f32_to_bf16_rows_kernel(const float* __restrict__ src, int64_t l
     }
 }
 
-// workspace: [0,256) ticket + item count; then the plan (one int2 per existing (sequence, query tile));
+// workspace: [0,256) ticket + item count; then the plan (one int4 per existing (sequence, query tile));
 // then, for fp32 tensors, their bf16 copies
 static size_t plan_entries(int64_t n, int S) { return (size_t)(n / kBM) + (size_t)S + 1; }
-static size_t plan_bytes(int64_t n, int S) { return align_up(plan_entries(n, S) * sizeof(int2), 256); }
+static size_t plan_bytes(int64_t n, int S) { return align_up(plan_entries(n, S) * sizeof(int4), 256); }
 size_t attention_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt) {
     size_t b = 256 + plan_bytes(n, S);
     if (dt != DASH_BF16) b += align_up((size_t)n * (Hq + 2 * Hkv) * D * 2, 256);
@@ -549,7 +549,7 @@ int attention_plan(const int32_t* cu_seqlens, int S, int64_t n, int Hq, void* ws
     if (n == 0) return DASH_OK;
     if (!ws || ((uintptr_t)ws % 256) || ws_bytes < 256 + plan_bytes(n, S)) return DASH_ERR_WORKSPACE;
     if ((int64_t)plan_entries(n, S) * Hq > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
-    attention_plan_kernel<<<1, 1024, 0, st>>>(cu_seqlens, S, Hq, (int2*)((char*)ws + 256), (int*)((char*)ws + 4), (unsigned int*)ws,
+    attention_plan_kernel<<<1, 1024, 0, st>>>(cu_seqlens, S, Hq, (int4*)((char*)ws + 256), (int*)((char*)ws + 4), (unsigned int*)ws,
                                               (int64_t)plan_entries(n, S));
     return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
@@ -622,7 +622,7 @@ static int attention_impl(const void* Q, const void* K, const void* V, void* O, 
     if (!p.status) return DASH_ERR_CUDA;
     p.ticket = (unsigned int*)ws;
     p.n_items = (const int*)((char*)ws + 4);
-    p.plan = (const int2*)((char*)ws + 256);
+    p.plan = (const int4*)((char*)ws + 256);
     if (!planned && (rc = attention_plan(cu_seqlens, S, n, Hq, ws, ws_bytes, st)) != DASH_OK) return rc;
     // persistent CTAs, two per SM, never more than there can be items
     int64_t grid64 = (int64_t)p.n_qtiles * Hq * S;
