@@ -422,12 +422,22 @@ def setup_sparse(args, dash, dev, rank):
     def norm():
         dash.dash_delta_norm(devt["U"], devt["H"], r_out=r, Hres_out=Ht, tau=state["tau"], cu_seqlens=cu, mask_out=mask)
 
+    indexed = bool(getattr(args, "indexed_attention", False))       # Q stays full-length and is fetched by index; only H~, K, V are compacted
+
     def compact():
-        dash.dash_compact(mask, cu, rows=[Ht, devt["Q"], devt["K"], devt["V"]], rows_out=outs, pos_in=pos, tok_in=tok, want_idx=False, ws=cws, outputs=o)
+        if indexed:
+            dash.dash_compact(mask, cu, rows=[Ht, devt["K"], devt["V"]], rows_out=[outs[0], outs[2], outs[3]], pos_in=pos, tok_in=tok, want_idx=False,
+                              ws=cws, outputs=o)
+        else:
+            dash.dash_compact(mask, cu, rows=[Ht, devt["Q"], devt["K"], devt["V"]], rows_out=outs, pos_in=pos, tok_in=tok, want_idx=False, ws=cws, outputs=o)
 
     def attn(max_len=None):
-        dash.dash_varlen_attention(outs[1].view(T, sh.Hq, sh.D), outs[2].view(T, sh.Hkv, sh.D), outs[3].view(T, sh.Hkv, sh.D), o["cu_out"],
-                                   max_len or state["max_len"], O=O, ws=attn_ws)
+        if indexed:
+            dash.dash_varlen_attention_indexed(devt["Q"].view(T, sh.Hq, sh.D), outs[2].view(T, sh.Hkv, sh.D), outs[3].view(T, sh.Hkv, sh.D), o["tok_out"],
+                                               o["cu_out"], max_len or state["max_len"], n=T, kv_packed=True, O=O, ws=attn_ws)
+        else:
+            dash.dash_varlen_attention(outs[1].view(T, sh.Hq, sh.D), outs[2].view(T, sh.Hkv, sh.D), outs[3].view(T, sh.Hkv, sh.D), o["cu_out"],
+                                       max_len or state["max_len"], O=O, ws=attn_ws)
 
     def step():                                   # no host synchronisation: the attention grid is sized by an upper bound
         norm(); compact(); attn(state["ub"])
@@ -447,17 +457,17 @@ def setup_sparse(args, dash, dev, rank):
     k = cu_out[-1]
     lens_out = [b - a for a, b in zip(cu_out[:-1], cu_out[1:])]
     state["max_len"] = max(1, max(lens_out))
-    row_b = (sh.d + (sh.Hq + 2 * sh.Hkv) * sh.D) * es
+    row_b = (sh.d + ((0 if indexed else sh.Hq) + 2 * sh.Hkv) * sh.D) * es
     which = "configs[3]: 131072 tokens, 20 % stay active" if args.workload == "cfg4" else "configs[4]: packed multimodal-shaped batch of 4 sequences"
     return {
-        "workload": f"{which}; Qwen2.5-7B layer shape, bf16; score+threshold -> compaction of H~,Q,K,V -> causal GQA attention over the "
-                    f"{k} active of {T} tokens (compacted lengths {lens_out})",
+        "workload": f"{which}; Qwen2.5-7B layer shape, bf16; score+threshold -> compaction of {'H~,K,V (Q fetched by index)' if indexed else 'H~,Q,K,V'} "
+                    f"-> causal GQA attention over the {k} active of {T} tokens (compacted lengths {lens_out})",
         "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 4,
-        "launch_note": "per step: delta_norm(+residual+threshold), compact (4 row tensors; + a memset of its look-back scratch), attention plan, attention",
+        "launch_note": f"per step: delta_norm(+residual+threshold), compact ({3 if indexed else 4} row tensors; + a memset of its look-back scratch), attention plan, attention",
         "h2d_bytes": _bytes(*host.values(), pos_host, cu_host), "d2h_bytes": _bytes(O_h, tok_h, cu_h, r_h),
         "extra": {"n_active_after": k, "tau": state["tau"]},
         "attn": (lambda: attn()), "attn_flops": attention_flops(cu_out, sh.Hq, sh.D),
-        "attn_name": f"attention_kernel<{sh.D}> over the compacted set",
+        "attn_name": f"attention_kernel<{sh.D}> over the compacted set" + (" (query tiles by index)" if indexed else ""),
         "norm": norm, "norm_bytes": T * (3 * sh.d * es + 5),
         "compact": compact, "compact_bytes": k * (2 * row_b + 16) + T * 9, "compact_rows": k, "row_bytes": row_b,
     }
@@ -852,6 +862,9 @@ def main():
     ap.add_argument("--seq", type=int, default=None, help="tokens per sequence (cfg1: 1024, cfg2: 8192, cfg3: 32768)")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--indexed-attention", action="store_true",
+                    help="cfg4 / cfg5: leave Q full-length and fetch its active rows by index in the attention kernel (dash_varlen_attention_indexed) "
+                         "instead of compacting Q")
     ap.add_argument("--library-gemms", action="store_true",
                     help="block steps use the library GEMMs (cuBLASLt) for the projections instead of this library's tcgen05 GEMMs with fused epilogues")
     args = ap.parse_args()

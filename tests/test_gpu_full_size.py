@@ -141,8 +141,12 @@ def _sparse_path(w, tau_from_oracle_K=None):
     cu_out_host = c["cu_out"].cpu()
     max_len = int((cu_out_host[1:] - cu_out_host[:-1]).max())
     O = dash.dash_varlen_attention(Qc, Kc, Vc, c["cu_out"], max(max_len, 1))
+    # the arrangement `bench.py --indexed-attention` times: Q left full-length, its active rows fetched by index (tok_out),
+    # K and V packed -- the same numbers bit for bit, so the oracle comparison of O below covers it too
+    O_idx = dash.dash_varlen_attention_indexed(Q, Kc, Vc, c["tok_out"], c["cu_out"], max(max_len, 1), n=T, kv_packed=True)
     torch.cuda.synchronize()
     assert dash.dash_check_status() == dash.OK
+    assert torch.equal(O[:k], O_idx[:k])
     return dict(r=r.cpu().numpy(), r_ref=r_ref, tau=tau, mask=mask.cpu().numpy(), m_ref=m_ref, c=c, k=k, O=O, Ht=Ht, Q=Q, K=K, V=V)
 
 
