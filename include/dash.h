@@ -103,8 +103,10 @@ typedef struct {
 /* r_out[t] = ||U_t||_2 / max(||H_t||_2, eps)  (REL)  or  ||U_t||_2  (ABS), fp32
  * accumulation.  U, H: [n, d] of type dt, d % 8 == 0.  If Hres_out != NULL the
  * residual update H~_t = H_t + U_t (Preliminaries) is written in the same pass
- * (may alias H).  If res_index != NULL (device int32 [n]), row t of the
- * residual is written to row res_index[t] of Hres_out instead of row t.
+ * (Hres_out may be H or U itself, same rows and stride).  If res_index != NULL
+ * (device int32 [n]), row t of the residual is written to row res_index[t] of
+ * Hres_out instead of row t; Hres_out must then overlap neither input
+ * (DASH_ERR_INVALID_ARG).
  * fused: NULL, or the threshold rule above.  n_dev: NULL, or a device int32
  * holding the true row count (<= n). */
 int dash_delta_norm(const void* U, const void* H, int64_t n, int d, int64_t ldU, int64_t ldH,
@@ -120,11 +122,11 @@ int dash_delta_norm(const void* U, const void* H, int64_t n, int d, int64_t ldU,
  * THRESHOLD_HALT_HIGH / KEEP_COUNT_HALT_HIGH: the same on -r (random halting needs no mode:
  *   pass random scores).
  * r: device fp32 [n]; cu_seqlens: device int32 [S+1] over the current packed
- * order; mask_out: device u8 [n] (1 = stays active). */
+ * order; mask_out: device u8 [n] (1 = stays active).  Needs no workspace (the
+ * radix select of the keep-count rule works in shared memory, one CTA per sequence). */
 int dash_select(const float* r, int64_t n, const int32_t* cu_seqlens, int S,
                 dash_sel_mode mode, float tau, const int32_t* keep_counts,
-                int keep_first, int keep_last, uint8_t* mask_out,
-                void* ws, size_t ws_bytes, void* stream);
+                int keep_first, int keep_last, uint8_t* mask_out, void* stream);
 
 /* ---- step 3: compaction / scatter (Sec. 3.4; Alg. 1 "gathering tokens") ---
  * One row tensor moved by the scan: dst[k] = src[idx[k]], rows of row_bytes
@@ -156,7 +158,7 @@ int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
  * forbids allocation calls on its worker threads (they synchronise the device).  (The
  * paper has no counterpart: it describes the method, not a memory policy.)
  * The look-back scratch lives in a fixed array inside the library instead, which every
- * GPU that loads the library holds until the process exits (256 KiB + 256 B).
+ * GPU that loads the library holds until the process exits (256 KiB + 512 B).
  *  - Limit: n <= DASH_COMPACT_STATIC_MAX_ROWS; larger inputs are rejected with
  *    DASH_ERR_TOO_LARGE before anything is enqueued.
  *  - Allocates nothing (no cudaMalloc / cudaFree, no allocating library routine); the
@@ -260,6 +262,15 @@ typedef struct {
                                     * 1 / rms, which the projection applies to its accumulators.  Needs fused_projections. */
 } dash_layer_cfg;
 
+/* LN of Eq. 1 is read as RMSNorm, y = x / rms(x) * w.  Its weight w can be folded, once and ahead of time, into the
+ * projection that follows the norm: W_out[i, j] = w[i] * W[i, j] for W, W_out [d, N] row-major of type dt (row strides ldw,
+ * ldo in elements, multiples of 16 bytes) and w [d] of type dt; the product is formed in fp32 and rounded once.  A block
+ * configured with rms_folded = 1 (rms2_folded = 1 for the norm in front of the FFN) expects such a matrix as Wqkv (Wgu): the
+ * norm then costs no pass of its own.  W_out may be W itself.  Asynchronous on `stream`.  DASH_ERR_INVALID_ARG for null or
+ * misaligned pointers, d < 1, N < 1, N not a multiple of 8 (bf16) / 4 (fp32), strides smaller than N. */
+int dash_fold_norm_weight(const void* W, const void* rms_weight, int d, int64_t N, int64_t ldw, dash_dtype dt,
+                          void* W_out, int64_t ldo, void* stream);
+
 /* Byte offsets of the intermediates inside the workspace of dash_layer_step
  * (for inspection by tests and tools).  Ht (H~ = H + U) is only written when the
  * halting rule is KEEP_COUNT or scatter_which is 0; with the threshold rule and
@@ -313,7 +324,7 @@ int dash_block_step(const dash_block_cfg* cfg, const void* H_in, const int32_t* 
                     void* ws, size_t ws_bytes, void* stream);
 
 /* ---- workspace sizes ------------------------------------------------------ */
-typedef enum { DASH_WS_SELECT = 0, DASH_WS_COMPACT = 1, DASH_WS_ATTENTION = 2, DASH_WS_DECODE = 3 } dash_ws_op;
+typedef enum { DASH_WS_COMPACT = 1, DASH_WS_ATTENTION = 2, DASH_WS_DECODE = 3 } dash_ws_op;
 /* n: rows allocated; S: sequences; Hq, Hkv, D, dt only matter for attention. */
 size_t dash_workspace_bytes(dash_ws_op op, int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt);
 

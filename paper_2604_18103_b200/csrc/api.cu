@@ -10,18 +10,17 @@ __device__ int g_status_word = 0;
 
 int* status_word_ptr() {
     // one address per device; looked up on first use with that device current
-    static int* ptrs[64] = {nullptr};
+    static std::atomic<int*> ptrs[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!ptrs[dev]) {
-        int* p = nullptr;
+    int* p = ptrs[dev].load(std::memory_order_acquire);
+    if (!p) {
         if (cudaGetSymbolAddress((void**)&p, g_status_word) != cudaSuccess) return nullptr;
-        ptrs[dev] = p;
+        ptrs[dev].store(p, std::memory_order_release);      // two threads that race here store the same address
     }
-    return ptrs[dev];
+    return p;
 }
 
-size_t select_ws_bytes(int64_t n, int S);
 size_t compact_ws_bytes_pub(int64_t n);
 size_t attention_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt);
 size_t decode_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D);
@@ -80,7 +79,6 @@ extern "C" double dash_flops_speedup(double n, double n_hat, int L, int l_s, dou
 extern "C" size_t dash_workspace_bytes(dash_ws_op op, int64_t n, int S, int Hq, int Hkv, int D, dash_dtype dt) {
     if (n < 0) return 0;
     switch (op) {
-        case DASH_WS_SELECT: return dash::select_ws_bytes(n, S);
         case DASH_WS_COMPACT: return dash::compact_ws_bytes_pub(n);
         case DASH_WS_ATTENTION: return dash::attention_ws_bytes(n, S, Hq, Hkv, D, dt);
         case DASH_WS_DECODE: return dash::decode_ws_bytes(n, S, Hq, Hkv, D);

@@ -534,11 +534,8 @@ template <int D, bool OUT_F32, bool GATHER>
 static int launch_attention(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p, int grid, cudaStream_t st) {
     using L = AttnSmem<D>;
     const int smem = L::kTotal + 1024;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(attention_kernel<D, OUT_F32, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (!set_max_smem_once(attention_kernel<D, OUT_F32, GATHER>, smem, configured)) return DASH_ERR_CUDA;
     return launch_pdl(attention_kernel<D, OUT_F32, GATHER>, grid, kAttnThreads, (size_t)smem, st, mq, mk, mv, p) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 

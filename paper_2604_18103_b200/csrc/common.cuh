@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "dash.h"
 
 #define DASH_CUDA_TRY(expr)                          \
@@ -28,6 +30,19 @@ inline int sm_count() {
     return sms > 0 ? sms : 148;
 }
 
+// cudaFuncAttributeMaxDynamicSharedMemorySize of `kernel`, set once per device: bit `device` of `done` remembers it (the call
+// is idempotent, so two threads that race here only repeat it)
+template <typename K>
+inline bool set_max_smem_once(K kernel, int smem_bytes, std::atomic<uint64_t>& done) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const uint64_t bit = (dev >= 0 && dev < 64) ? (1ull << dev) : 0ull;
+    if (bit && (done.load(std::memory_order_acquire) & bit)) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return false;
+    if (bit) done.fetch_or(bit, std::memory_order_release);
+    return true;
+}
+
 // Launch of a kernel that calls pdl_wait() before its first global access: it may start while the kernel in front of it in
 // the stream drains (programmatic dependent launch); behind anything else it is an ordinary launch.
 template <typename... KArgs, typename... Args>
@@ -49,6 +64,12 @@ __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+// coherent 128-bit load: for data that this very launch may also write (an output that aliases an input)
+__device__ __forceinline__ uint4 ld_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ void st_v4(void* p, uint4 v) {

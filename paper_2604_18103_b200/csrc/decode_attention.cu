@@ -501,11 +501,8 @@ static int launch_decode(const CUtensorMap& mq, const CUtensorMap& mk, const CUt
                          cudaStream_t st) {
     using L = DecSmem<D>;
     const int smem = L::kTotal + 1024;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (!set_max_smem_once(decode_kernel<D>, smem, configured)) return DASH_ERR_CUDA;
     return launch_pdl(decode_kernel<D>, grid, kDecThreads, (size_t)smem, st, mq, mk, mv, p, box_heads) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }
 

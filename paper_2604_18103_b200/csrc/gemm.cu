@@ -257,7 +257,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     if (live) {
 #pragma unroll
                         for (int e = 0; e < 32; e += 8) {
-                            const uint4 hv = ld_nc_v4(hsrc + c * 32 + e);
+                            const uint4 hv = ld_v4(hsrc + c * 32 + e);        // coherent: x_full may be H itself (identity token rows)
                             const float hf[8] = {bf16lo(hv.x), bf16hi(hv.x), bf16lo(hv.y), bf16hi(hv.y), bf16lo(hv.z), bf16hi(hv.z), bf16lo(hv.w), bf16hi(hv.w)};
                             float y[8];
 #pragma unroll
@@ -371,11 +371,8 @@ static int make_map_2d_bf16(CUtensorMap* map, const void* basep, uint64_t inner,
 template <int EPI>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mw, const GemmArgs& g, cudaStream_t st) {
     const int smem = kGStages * kGStageBytes + 1024 + 256;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return DASH_ERR_CUDA;
-        configured = true;
-    }
+    static std::atomic<uint64_t> configured{0};
+    if (!set_max_smem_once(gemm_kernel<EPI>, smem, configured)) return DASH_ERR_CUDA;
     const int tiles = ((g.n + 2 * kGM - 1) / (2 * kGM)) * g.n_tiles;
     int pairs = sm_count() / 2;
     if (pairs > tiles) pairs = tiles;

@@ -1,6 +1,7 @@
 // HBM-bound kernels of the halted-prefill path: delta-attention score (+ fused
 // residual and threshold), halting rule, single-pass compaction, scatter.
 #include "common.cuh"
+#include "dash_testing.h"
 #include "sm100_ptx.cuh"
 
 namespace dash {
@@ -52,7 +53,7 @@ __global__ void __launch_bounds__(256)
 delta_norm_kernel(const char* __restrict__ U, const char* __restrict__ H, int64_t n, int nvec,
                   int64_t ldU_b, int64_t ldH_b, int mode, float eps, float* __restrict__ r_out,
                   char* Hres, int64_t ldR_b, const int32_t* __restrict__ res_index,
-                  FusedThreshold ft, const int32_t* __restrict__ n_dev) {
+                  FusedThreshold ft, const int32_t* __restrict__ n_dev, int aliased) {
     const int lane = threadIdx.x & 31;
     const int wpb = blockDim.x >> 5;
     if (n_dev) { int64_t nd = *n_dev; if (nd < n) n = nd; }
@@ -70,8 +71,10 @@ delta_norm_kernel(const char* __restrict__ U, const char* __restrict__ H, int64_
             for (int k = 0; k < CH; ++k) {
                 int v = base + k * 32 + lane;
                 if (v < nvec) {
-                    a[k] = ld_nc_v4(u + ((int64_t)v << 4));
-                    if (need_h) b[k] = ld_nc_v4(h + ((int64_t)v << 4));
+                    // the read-only path only where the residual output overlaps neither input (each vector is read before it is
+                    // written, by the same thread, so an output that is H itself is well defined -- through coherent loads)
+                    a[k] = aliased ? ld_v4(u + ((int64_t)v << 4)) : ld_nc_v4(u + ((int64_t)v << 4));
+                    if (need_h) b[k] = aliased ? ld_v4(h + ((int64_t)v << 4)) : ld_nc_v4(h + ((int64_t)v << 4));
                 }
             }
 #pragma unroll
@@ -262,7 +265,7 @@ compact_kernel(const uint8_t* __restrict__ mask, int64_t n_upper, const int32_t*
                RowStreams rs, const int32_t* __restrict__ pos_in, int32_t* __restrict__ pos_out,
                const int32_t* __restrict__ tok_in, int32_t* __restrict__ tok_out,
                int32_t* __restrict__ idx_out, int32_t* __restrict__ cu_out, int32_t* __restrict__ n_out_dev,
-               unsigned long long* tile_state, unsigned int* ticket, int* status, int mask_vec16) {
+               unsigned long long* tile_state, unsigned int* ticket, int* status, int mask_vec16, uint32_t spin_limit) {
     constexpr int NW = TILE / 32;                       // warps that ballot
     constexpr int NWARPS = kCompactThreads / 32;
     __shared__ unsigned int s_ballot[NW];
@@ -342,7 +345,7 @@ compact_kernel(const uint8_t* __restrict__ mask, int64_t n_upper, const int32_t*
                 if (j >= 0) {
                     st = ld_state(&tile_state[j]);
                     while ((st >> 32) == 0) {
-                        if (++spins > kSpinLimit) { timed_out = true; break; }
+                        if (++spins > spin_limit) { timed_out = true; break; }
                         __nanosleep(32);
                         st = ld_state(&tile_state[j]);
                     }
@@ -635,20 +638,26 @@ extern "C" int dash_delta_norm(const void* U, const void* H, int64_t n, int d, i
     const int nvec = d * es / 16;
     cudaStream_t st = (cudaStream_t)stream;
     const int grid = rows_grid(n, 8);
+    // does the residual output overlap an input?  (H~ written over H is allowed when row t goes to row t)
+    auto overlaps = [&](const void* a, int64_t lda) {
+        if (!Hres_out || !a) return false;
+        const char *a0 = (const char*)a, *a1 = a0 + n * lda * es, *o0 = (const char*)Hres_out, *o1 = o0 + n * ldHres * es;
+        return a0 < o1 && o0 < a1;
+    };
+    const int aliased = (overlaps(U, ldU) || overlaps(H, ldH)) ? 1 : 0;
+    if (aliased && res_index) return DASH_ERR_INVALID_ARG;      // an indexed destination inside an input would be read after it was written
     if (dt == DASH_BF16)
         delta_norm_kernel<true><<<grid, 256, 0, st>>>((const char*)U, (const char*)H, n, nvec, ldU * es, ldH * es, (int)mode, eps,
-                                                      r_out, (char*)Hres_out, ldHres * es, res_index, ft, n_dev);
+                                                      r_out, (char*)Hres_out, ldHres * es, res_index, ft, n_dev, aliased);
     else
         delta_norm_kernel<false><<<grid, 256, 0, st>>>((const char*)U, (const char*)H, n, nvec, ldU * es, ldH * es, (int)mode, eps,
-                                                       r_out, (char*)Hres_out, ldHres * es, res_index, ft, n_dev);
+                                                       r_out, (char*)Hres_out, ldHres * es, res_index, ft, n_dev, aliased);
     DASH_CUDA_TRY(cudaGetLastError());
     return DASH_OK;
 }
 
 extern "C" int dash_select(const float* r, int64_t n, const int32_t* cu_seqlens, int S, dash_sel_mode mode, float tau,
-                           const int32_t* keep_counts, int keep_first, int keep_last, uint8_t* mask_out,
-                           void* ws, size_t ws_bytes, void* stream) {
-    (void)ws; (void)ws_bytes;
+                           const int32_t* keep_counts, int keep_first, int keep_last, uint8_t* mask_out, void* stream) {
     if (n < 0 || S < 1 || !cu_seqlens || keep_first < 0 || keep_last < 0) return DASH_ERR_INVALID_ARG;
     if (mode < DASH_SEL_THRESHOLD || mode > DASH_SEL_KEEP_COUNT_HALT_HIGH) return DASH_ERR_INVALID_ARG;
     const int halt_high = (mode == DASH_SEL_THRESHOLD_HALT_HIGH || mode == DASH_SEL_KEEP_COUNT_HALT_HIGH) ? 1 : 0;
@@ -710,11 +719,12 @@ static size_t compact_ws_bytes(int64_t n) {
     return align_up(256 + (size_t)tiles * 8, 256);
 }
 
-extern "C" int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
-                            const dash_rows* rows, int n_rows,
-                            const int32_t* pos_in, int32_t* pos_out, const int32_t* tok_in, int32_t* tok_out,
-                            int32_t* idx_out, int32_t* cu_out, int32_t* n_out_dev,
-                            void* ws, size_t ws_bytes, void* stream) {
+// stall: test hook (see dash_testing.h) -- look-back path whatever the size, tile ticket started at 1, spin limit as given
+static int compact_impl(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
+                        const dash_rows* rows, int n_rows,
+                        const int32_t* pos_in, int32_t* pos_out, const int32_t* tok_in, int32_t* tok_out,
+                        int32_t* idx_out, int32_t* cu_out, int32_t* n_out_dev,
+                        void* ws, size_t ws_bytes, void* stream, bool stall, uint32_t spin_limit) {
     if (n < 0 || S < 1 || !cu_in || !cu_out || n_rows < 0 || n_rows > DASH_MAX_ROW_STREAMS) return DASH_ERR_INVALID_ARG;
     if (n > 0 && !mask) return DASH_ERR_INVALID_ARG;
     if (n_rows > 0 && !rows) return DASH_ERR_INVALID_ARG;
@@ -735,16 +745,17 @@ extern "C" int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in
     cudaStream_t st = (cudaStream_t)stream;
     const int TILE = compact_tile_for(n);
     const int tiles = (int)((n + TILE - 1) / TILE) > 0 ? (int)((n + TILE - 1) / TILE) : 1;
-    const bool direct = n <= kCompactDirectMaxRows;
+    const bool direct = n <= kCompactDirectMaxRows && !stall;
     unsigned int* ticket = (unsigned int*)ws;
     unsigned long long* state = (unsigned long long*)((char*)ws + 256);
     if (!direct) DASH_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)tiles * 8, st));
+    if (stall) DASH_CUDA_TRY(cudaMemsetAsync(ws, 1, 1, st));          // ticket = 1: tile 0 is never taken, tile 1 waits for it in vain
     int* status = status_word_ptr();
     if (!status) return DASH_ERR_CUDA;
     const int mask_vec16 = aligned16(mask) ? 1 : 0;
 #define DASH_LAUNCH_COMPACT(T, DIRECT)                                                                                       \
     compact_kernel<T, DIRECT><<<tiles, kCompactThreads, 0, st>>>(mask, n, cu_in, S, rs, pos_in, pos_out, tok_in, tok_out, \
-                                                                 idx_out, cu_out, n_out_dev, state, ticket, status, mask_vec16)
+                                                                 idx_out, cu_out, n_out_dev, state, ticket, status, mask_vec16, spin_limit)
     if (direct) {
         switch (TILE) {
             case 256: DASH_LAUNCH_COMPACT(256, true); break;
@@ -763,6 +774,22 @@ extern "C" int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in
 #undef DASH_LAUNCH_COMPACT
     DASH_CUDA_TRY(cudaGetLastError());
     return DASH_OK;
+}
+
+extern "C" int dash_compact(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
+                            const dash_rows* rows, int n_rows,
+                            const int32_t* pos_in, int32_t* pos_out, const int32_t* tok_in, int32_t* tok_out,
+                            int32_t* idx_out, int32_t* cu_out, int32_t* n_out_dev,
+                            void* ws, size_t ws_bytes, void* stream) {
+    return compact_impl(mask, n, cu_in, S, rows, n_rows, pos_in, pos_out, tok_in, tok_out, idx_out, cu_out, n_out_dev, ws, ws_bytes, stream, false,
+                        kSpinLimit);
+}
+
+extern "C" int dash_testing_compact_stalled(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S, int32_t* idx_out, int32_t* cu_out,
+                                            int32_t* n_out_dev, uint32_t spin_limit, void* ws, size_t ws_bytes, void* stream) {
+    if (n < 64 || spin_limit < 1 || spin_limit > kSpinLimit) return DASH_ERR_INVALID_ARG;
+    return compact_impl(mask, n, cu_in, S, nullptr, 0, nullptr, nullptr, nullptr, nullptr, idx_out, cu_out, n_out_dev, ws, ws_bytes, stream, true,
+                        spin_limit);
 }
 
 extern "C" int dash_scatter(const void* src, int64_t n, int64_t row_bytes, int64_t src_ld_bytes,
@@ -790,15 +817,15 @@ static __device__ __align__(256) unsigned char g_compact_scratch[(kStaticScratch
 // Host code cannot use the array's name as a pointer (on the host it is only a handle for
 // the runtime): ask for its device address once per device, with that device current.
 static void* compact_scratch_ptr() {
-    static void* ptrs[64] = {nullptr};
+    static std::atomic<void*> ptrs[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!ptrs[dev]) {
-        void* p = nullptr;
+    void* p = ptrs[dev].load(std::memory_order_acquire);
+    if (!p) {
         if (cudaGetSymbolAddress((void**)&p, g_compact_scratch) != cudaSuccess) return nullptr;
-        ptrs[dev] = p;
+        ptrs[dev].store(p, std::memory_order_release);      // two threads that race here store the same address
     }
-    return ptrs[dev];
+    return p;
 }
 
 extern "C" int dash_compact_static(const uint8_t* mask, int64_t n, const int32_t* cu_in, int S,
@@ -814,7 +841,6 @@ extern "C" int dash_compact_static(const uint8_t* mask, int64_t n, const int32_t
 }
 
 namespace dash {
-size_t select_ws_bytes(int64_t, int) { return 256; }
 
 // r (and, with ft.mask_out set, the threshold decision) from the per-row partial sums of the output-projection epilogue; with
 // inv_rms_out set also the row factor of the next RMSNorm, 1 / sqrt(mean((h+u)^2) + rms_eps)

@@ -225,6 +225,28 @@ swiglu_kernel(const char* __restrict__ GU, int64_t ldgu_b, char* __restrict__ AC
     }
 }
 
+// W_out[i, :] = w[i] * W[i, :]: the norm's weight folded into the projection behind it (one 16-byte vector per thread)
+template <bool BF16>
+__global__ void __launch_bounds__(256)
+fold_norm_weight_kernel(const char* __restrict__ W, int64_t ldw_b, const char* __restrict__ w, char* __restrict__ Wout, int64_t ldo_b, int d, int vpr) {
+    const int64_t total = (int64_t)d * vpr;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int row = (int)(i / vpr), v = (int)(i - (int64_t)row * vpr);
+        const uint4 a = *reinterpret_cast<const uint4*>(W + row * ldw_b + ((int64_t)v << 4));
+        uint4 o;
+        if (BF16) {
+            const float g = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(w)[row]);
+            o.x = pack_bf16(bf16lo(a.x) * g, bf16hi(a.x) * g); o.y = pack_bf16(bf16lo(a.y) * g, bf16hi(a.y) * g);
+            o.z = pack_bf16(bf16lo(a.z) * g, bf16hi(a.z) * g); o.w = pack_bf16(bf16lo(a.w) * g, bf16hi(a.w) * g);
+        } else {
+            const float g = reinterpret_cast<const float*>(w)[row];
+            o.x = __float_as_uint(__uint_as_float(a.x) * g); o.y = __float_as_uint(__uint_as_float(a.y) * g);
+            o.z = __float_as_uint(__uint_as_float(a.z) * g); o.w = __float_as_uint(__uint_as_float(a.w) * g);
+        }
+        *reinterpret_cast<uint4*>(Wout + row * ldo_b + ((int64_t)v << 4)) = o;
+    }
+}
+
 static bool cfg_ok(const dash_layer_cfg* c) {
     if (!c || c->d <= 0 || c->Hq < 1 || c->Hkv < 1 || (c->D != 64 && c->D != 128)) return false;
     if ((c->d % 8) || (c->Hq % c->Hkv)) return false;
@@ -244,6 +266,23 @@ static bool cfg_ok(const dash_layer_cfg* c) {
 }  // namespace dash
 
 using namespace dash;
+
+extern "C" int dash_fold_norm_weight(const void* W, const void* rms_weight, int d, int64_t N, int64_t ldw, dash_dtype dt,
+                                     void* W_out, int64_t ldo, void* stream) {
+    if (dt != DASH_F32 && dt != DASH_BF16) return DASH_ERR_INVALID_ARG;
+    const int es = dt == DASH_BF16 ? 2 : 4, epv = 16 / es;
+    if (!W || !rms_weight || !W_out || d < 1 || N < 1 || (N % epv) || ldw < N || ldo < N) return DASH_ERR_INVALID_ARG;
+    if (!aligned16(W) || !aligned16(W_out) || (ldw * es) % 16 || (ldo * es) % 16 || ((uintptr_t)rms_weight % es)) return DASH_ERR_INVALID_ARG;
+    const int64_t vpr = N / epv;
+    if (vpr > 0x7fffffffLL) return DASH_ERR_UNSUPPORTED;
+    int64_t blocks = ((int64_t)d * vpr + 255) / 256, cap = (int64_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dt == DASH_BF16) fold_norm_weight_kernel<true><<<(int)blocks, 256, 0, st>>>((const char*)W, ldw * es, (const char*)rms_weight, (char*)W_out, ldo * es, d, (int)vpr);
+    else fold_norm_weight_kernel<false><<<(int)blocks, 256, 0, st>>>((const char*)W, ldw * es, (const char*)rms_weight, (char*)W_out, ldo * es, d, (int)vpr);
+    DASH_CUDA_TRY(cudaGetLastError());
+    return DASH_OK;
+}
 
 extern "C" int dash_layer_workspace(const dash_layer_cfg* cfg, int64_t n, int S, dash_layer_ws_layout* out) {
     if (!cfg_ok(cfg) || n < 0 || S < 1 || !out) return DASH_ERR_INVALID_ARG;
@@ -382,8 +421,7 @@ static int score_and_select(const dash_layer_cfg* cfg, const void* H_in, const i
                              cfg->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr, cu_in + S, st);
     if (rc != DASH_OK) return rc;
     if (cfg->sel_mode != DASH_SEL_THRESHOLD)
-        rc = dash_select(r_out, n, cu_in, S, cfg->sel_mode, cfg->tau, cfg->keep_counts, cfg->keep_first, cfg->keep_last, mask_out,
-                         nullptr, 0, st);
+        rc = dash_select(r_out, n, cu_in, S, cfg->sel_mode, cfg->tau, cfg->keep_counts, cfg->keep_first, cfg->keep_last, mask_out, st);
     return rc;
 }
 
@@ -504,7 +542,7 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         if ((rc = launch_sums_to_score(W.sums, d / 256, n, a->norm_mode, a->norm_eps, r_out, a->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr,
                                        n_dev, have_inv_rms2 ? W.inv_rms2 : nullptr, d, a->rms_eps, st)) != DASH_OK) return rc;
         if (a->sel_mode != DASH_SEL_THRESHOLD &&
-            (rc = dash_select(r_out, n, cu_in, S, a->sel_mode, a->tau, a->keep_counts, a->keep_first, a->keep_last, mask_out, nullptr, 0, st)) != DASH_OK)
+            (rc = dash_select(r_out, n, cu_in, S, a->sel_mode, a->tau, a->keep_counts, a->keep_first, a->keep_last, mask_out, st)) != DASH_OK)
             return rc;
     } else if (rc == DASH_ERR_UNSUPPORTED) {
         if ((rc = out_proj_U(a, cu_in, S, n, W, st)) != DASH_OK) return rc;
@@ -541,7 +579,7 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
                              a->sel_mode == DASH_SEL_THRESHOLD ? &ft : nullptr, n_dev, st);
         if (rc != DASH_OK) return rc;
         if (a->sel_mode != DASH_SEL_THRESHOLD &&
-            (rc = dash_select(r_out, n, cu_in, S, a->sel_mode, a->tau, a->keep_counts, a->keep_first, a->keep_last, mask_out, nullptr, 0, st)) != DASH_OK)
+            (rc = dash_select(r_out, n, cu_in, S, a->sel_mode, a->tau, a->keep_counts, a->keep_first, a->keep_last, mask_out, st)) != DASH_OK)
             return rc;
     }
     // H' = H~ + F to x_full (every entering token: H' is also the last updated value of the tokens that halt here) and,

@@ -2,7 +2,8 @@
 
 Argument marshalling only: every step of the path runs in the library's
 kernels.  Tensors are torch CUDA tensors (torch provides device memory and the
-current stream); nothing here computes on the host.  If the library cannot be
+current stream); the only tensor operations here move data (concatenating the
+Q | K | V and gate | up weight matrices, copies to the device) -- no arithmetic.  If the library cannot be
 loaded the import of a symbol raises -- there is no CPU fallback.
 """
 from __future__ import annotations
@@ -19,7 +20,7 @@ F32, BF16 = 0, 1
 NORM_REL, NORM_ABS = 0, 1
 SEL_THRESHOLD, SEL_KEEP_COUNT, SEL_THRESHOLD_HALT_HIGH, SEL_KEEP_COUNT_HALT_HIGH = 0, 1, 2, 3
 SIGNAL_ATTN, SIGNAL_BLOCK = 0, 1
-WS_SELECT, WS_COMPACT, WS_ATTENTION, WS_DECODE = 0, 1, 2, 3
+WS_COMPACT, WS_ATTENTION, WS_DECODE = 1, 2, 3
 OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -30,8 +31,9 @@ EXPORTS = [
     "dash_delta_norm", "dash_select", "dash_compact", "dash_scatter", "dash_varlen_attention",
     "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes", "dash_compact_static",
     "dash_block_workspace", "dash_block_step", "dash_decode_attention", "dash_varlen_attention_indexed",
-    "dash_keep_counts_device",
+    "dash_keep_counts_device", "dash_fold_norm_weight",
 ]
+TEST_HOOKS = ["dash_testing_compact_stalled"]        # include/dash_testing.h
 COMPACT_STATIC_MAX_ROWS = 1 << 20
 
 
@@ -89,7 +91,7 @@ def lib() -> ctypes.CDLL:
         L.dash_delta_norm.argtypes = [c_void_p, c_void_p, c_int64, c_int, c_int64, c_int64, c_int, c_int, c_float,
                                       c_void_p, c_void_p, c_int64, c_void_p, POINTER(Threshold), c_void_p, c_void_p]
         L.dash_select.argtypes = [c_void_p, c_int64, c_void_p, c_int, c_int, c_float, c_void_p, c_int, c_int,
-                                  c_void_p, c_void_p, c_size_t, c_void_p]
+                                  c_void_p, c_void_p]
         L.dash_compact.argtypes = [c_void_p, c_int64, c_void_p, c_int, POINTER(Rows), c_int, c_void_p, c_void_p,
                                    c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.dash_compact_static.argtypes = [c_void_p, c_int64, c_void_p, c_int, POINTER(Rows), c_int, c_void_p, c_void_p,
@@ -103,6 +105,7 @@ def lib() -> ctypes.CDLL:
                                                                                   c_int, c_int, c_int, c_float, c_int, c_int,
                                                                                   c_void_p, c_size_t, c_void_p]
         L.dash_keep_counts_device.argtypes = [c_void_p, c_int, c_double, c_int, c_int, c_int, c_void_p, c_void_p]
+        L.dash_fold_norm_weight.argtypes = [c_void_p, c_void_p, c_int, c_int64, c_int64, c_int, c_void_p, c_int64, c_void_p]
         L.dash_layer_workspace.argtypes = [POINTER(LayerCfg), c_int64, c_int, POINTER(LayerWsLayout)]
         L.dash_layer_step.argtypes = [POINTER(LayerCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -113,6 +116,8 @@ def lib() -> ctypes.CDLL:
         L.dash_block_step.argtypes = [POINTER(BlockCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_size_t, c_void_p]
+        L.dash_testing_compact_stalled.argtypes = [c_void_p, c_int64, c_void_p, c_int, c_void_p, c_void_p, c_void_p, ctypes.c_uint32,
+                                                   c_void_p, c_size_t, c_void_p]
         L.dash_workspace_bytes.restype = c_size_t
         L.dash_workspace_bytes.argtypes = [c_int, c_int64, c_int, c_int, c_int, c_int, c_int]
         _lib = L
@@ -207,7 +212,7 @@ def dash_select(r: torch.Tensor, cu_seqlens: torch.Tensor, mode: int, tau: float
     if mask_out is None:
         mask_out = torch.empty(n, dtype=torch.uint8, device=r.device)
     st = lib().dash_select(_p(r), n, _p(cu_seqlens), cu_seqlens.numel() - 1, mode, tau, _p(keep_counts), keep_first, keep_last,
-                           _p(mask_out), None, 0, _stream())
+                           _p(mask_out), _stream())
     _check(st, "dash_select")
     return mask_out
 
@@ -262,6 +267,20 @@ def dash_compact(mask: torch.Tensor, cu_in: torch.Tensor, rows: Sequence[torch.T
                             _p(idx), _p(cu_out), _p(n_out), _p(ws), ws.numel(), _stream())
     _check(st, "dash_compact")
     return {"idx": idx, "cu_out": cu_out, "n_out": n_out, "rows": list(rows_out), "pos_out": pos_out, "tok_out": tok_out}
+
+
+def dash_testing_compact_stalled(mask: torch.Tensor, cu_in: torch.Tensor, spin_limit: int = 1000):
+    """Test hook (include/dash_testing.h): the look-back compaction with tile 0 never taken, so that a bounded device-side
+    wait runs out.  Returns dict(idx, cu_out, n_out); the device status word then holds DASH_ERR_TIMEOUT."""
+    _dev(mask, cu_in)
+    n, S, dev = mask.numel(), cu_in.numel() - 1, mask.device
+    idx = torch.zeros(n, dtype=torch.int32, device=dev)
+    cu_out = torch.zeros(S + 1, dtype=torch.int32, device=dev)
+    n_out = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = workspace(dash_workspace_bytes(WS_COMPACT, n, S), dev)
+    st = lib().dash_testing_compact_stalled(_p(mask), n, _p(cu_in), S, _p(idx), _p(cu_out), _p(n_out), int(spin_limit), _p(ws), ws.numel(), _stream())
+    _check(st, "dash_testing_compact_stalled")
+    return {"idx": idx, "cu_out": cu_out, "n_out": n_out}
 
 
 def dash_scatter(src: torch.Tensor, dst_full: torch.Tensor, tok_index: Optional[torch.Tensor] = None,
@@ -347,6 +366,16 @@ def dash_decode_attention(q: torch.Tensor, Kc: torch.Tensor, Vc: torch.Tensor, c
 
 
 # ---- the block step ---------------------------------------------------------------
+def dash_fold_norm_weight(W: torch.Tensor, rms_weight: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """W_out[i, :] = rms_weight[i] * W[i, :] on the device (the norm's weight folded into the projection behind it)."""
+    _dev(W, rms_weight, out)
+    if out is None:
+        out = torch.empty_like(W)
+    st = lib().dash_fold_norm_weight(_p(W), _p(rms_weight), W.shape[0], W.shape[1], W.stride(0), dtype_code(W), _p(out), out.stride(0), _stream())
+    _check(st, "dash_fold_norm_weight")
+    return out
+
+
 def _projections_fit(shape) -> bool:
     """True if this library's GEMMs take every projection of the block (256-column tiles, depth in steps of 64)."""
     nq, hd = (shape.Hq + 2 * shape.Hkv) * shape.D, shape.Hq * shape.D
@@ -360,15 +389,14 @@ class Layer:
     def __init__(self, shape, weights, device, norm_mode=NORM_REL, norm_eps=1e-12, sel_mode=SEL_THRESHOLD, tau=0.0,
                  keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2, fused_projections=True):
         self.shape = shape
-        Wqkv = torch.cat([weights["Wq"], weights["Wk"], weights["Wv"]], dim=1)
-        # with fused projections (bf16) the norm's weight is folded into the projection once, here: the library then needs no
-        # normalisation pass (the row factor 1 / rms is applied to the projection's accumulators)
-        self.rms_folded = bool(fused_projections) and Wqkv.dtype == torch.bfloat16 and _projections_fit(shape)
-        if self.rms_folded:
-            Wqkv = (weights["rms_w"].float()[:, None] * Wqkv.float()).to(Wqkv.dtype)
-        self.Wqkv = Wqkv.contiguous().to(device)
+        self.Wqkv = torch.cat([weights["Wq"], weights["Wk"], weights["Wv"]], dim=1).contiguous().to(device)
         self.Wo = weights["Wo"].contiguous().to(device)
         self.rms_w = weights["rms_w"].contiguous().to(device)
+        # with fused projections (bf16) the norm's weight is folded into the projection once, here, by the library: the step then
+        # needs no normalisation pass (the row factor 1 / rms is applied to the projection's accumulators)
+        self.rms_folded = bool(fused_projections) and self.Wqkv.dtype == torch.bfloat16 and _projections_fit(shape)
+        if self.rms_folded:
+            dash_fold_norm_weight(self.Wqkv, self.rms_w, out=self.Wqkv)
         self.keep_counts = keep_counts
         self.cfg = LayerCfg(shape.d, shape.Hq, shape.Hkv, shape.D, dtype_code(self.Wo), self.Wqkv.data_ptr(), self.Wo.data_ptr(),
                             self.rms_w.data_ptr(), shape.rms_eps, shape.rope_base, norm_mode, norm_eps, sel_mode, tau,
@@ -406,13 +434,12 @@ class Block:
     def __init__(self, shape, weights, device, signal=SIGNAL_ATTN, **layer_kwargs):
         self.layer = Layer(shape, weights, device, **layer_kwargs)
         self.shape = shape
-        Wgu = torch.cat([weights["Wg"], weights["Wu"]], dim=1)
-        self.rms2_folded = self.layer.rms_folded and signal == SIGNAL_ATTN
-        if self.rms2_folded:
-            Wgu = (weights["rms2_w"].float()[:, None] * Wgu.float()).to(Wgu.dtype)
-        self.Wgu = Wgu.contiguous().to(device)
+        self.Wgu = torch.cat([weights["Wg"], weights["Wu"]], dim=1).contiguous().to(device)
         self.Wd = weights["Wd"].contiguous().to(device)
         self.rms2_w = weights["rms2_w"].contiguous().to(device)
+        self.rms2_folded = self.layer.rms_folded and signal == SIGNAL_ATTN
+        if self.rms2_folded:
+            dash_fold_norm_weight(self.Wgu, self.rms2_w, out=self.Wgu)
         self.cfg = BlockCfg(self.layer.cfg, shape.m, self.Wgu.data_ptr(), self.Wd.data_ptr(), self.rms2_w.data_ptr(), signal, int(self.rms2_folded))
 
     def set_tau(self, tau: float):

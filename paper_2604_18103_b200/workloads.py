@@ -231,30 +231,36 @@ def random_mask(n: int, keep_prob: float, seed: int, stream: int = 30) -> torch.
 
 
 def sample_rows(cu: torch.Tensor, n_samples: int, seed: int, tile: int = 128) -> torch.Tensor:
-    """Seeded sample of packed row indices that always holds the first and last
-    row of every sequence and the rows on both sides of every `tile` boundary
-    (counted from the start of the sequence), padded with uniform draws."""
-    picks = set()
-    for s in range(cu.numel() - 1):
-        a, b = int(cu[s]), int(cu[s + 1])
-        if b <= a:
-            continue
-        picks.update((a, b - 1))
-    T = int(cu[-1])
+    """Seeded sample of packed row indices for checks that cannot visit every row.  In this order, as far as the budget
+    n_samples goes: the first and last row of every sequence; one row drawn inside every `tile`-row tile of every sequence
+    (tiles counted from the start of the sequence), so that no tile goes unvisited; the rows on both sides of every tile
+    boundary; uniform draws over all rows."""
     g = _gen(seed, 31)
-    bounds = []
-    for s in range(cu.numel() - 1):
-        a, b = int(cu[s]), int(cu[s + 1])
-        for t in range(a + tile, b, tile):
-            bounds.extend((t - 1, t))
-    if bounds:
-        bt = torch.tensor(bounds)
-        budget = max(0, n_samples // 2)
-        if bt.numel() > budget:
-            sel = torch.randperm(bt.numel(), generator=g)[:budget]
-            bt = bt[sel]
-        picks.update(int(x) for x in bt)
-    if T > 0:
-        extra = torch.randint(0, T, (max(0, n_samples - len(picks)),), generator=g)
-        picks.update(int(x) for x in extra)
+    picks: List[int] = []
+    seen = set()
+
+    def add(rows) -> None:
+        for r in rows:
+            r = int(r)
+            if r not in seen and len(picks) < n_samples:
+                seen.add(r)
+                picks.append(r)
+
+    S = cu.numel() - 1
+    bounds = [(int(cu[s]), int(cu[s + 1])) for s in range(S) if int(cu[s + 1]) > int(cu[s])]
+    for a, b in bounds:
+        add((a, b - 1))
+    starts = [(t, min(t + tile, b)) for a, b in bounds for t in range(a, b, tile)]
+    if starts:
+        u = torch.rand(len(starts), generator=g)
+        order = torch.randperm(len(starts), generator=g).tolist()         # if the budget is short, the tiles left out are random ones
+        add(starts[i][0] + int(float(u[i]) * (starts[i][1] - starts[i][0])) for i in order)
+    edges = [r for a, b in bounds for t in range(a + tile, b, tile) for r in (t - 1, t)]
+    if edges:
+        order = torch.randperm(len(edges) // 2, generator=g).tolist()
+        add(r for i in order for r in edges[2 * i:2 * i + 2])
+    T = int(cu[-1])
+    if T > 0 and len(picks) < min(n_samples, T):
+        extra = torch.randperm(T, generator=g) if T <= 4 * n_samples else torch.randint(0, T, (4 * n_samples,), generator=g)
+        add(extra.tolist())
     return torch.tensor(sorted(picks), dtype=torch.int64)

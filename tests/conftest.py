@@ -24,3 +24,25 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+# ---- measured error ratios of the full-size parity tests, written where a GPU run's artefacts go ----
+_ERRORS = {}
+
+
+def record_error(name, err_over_tensor_rms, err_over_row_rms):
+    """max |err| / RMS(reference tensor) and the worst row's max |err| / RMS(that row), for the record."""
+    _ERRORS[name] = {"max_err_over_tensor_rms": err_over_tensor_rms, "max_err_over_row_rms": err_over_row_rms}
+
+
+def pytest_sessionfinish(session, exitstatus):
+    if not _ERRORS:
+        return
+    import json
+    out = os.path.join(ROOT, "gpurun_out")
+    try:
+        os.makedirs(out, exist_ok=True)
+        with open(os.path.join(out, "parity_errors.json"), "w") as f:
+            json.dump(_ERRORS, f, indent=1, sort_keys=True)
+    except OSError:
+        pass

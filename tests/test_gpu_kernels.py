@@ -75,6 +75,59 @@ def test_delta_norm_matches_oracle(dtype, n, d):
         assert torch.equal(full[perm.long().to(DEV)], ref)
 
 
+def test_delta_norm_residual_written_over_an_input():
+    """H~ = H + U written over H itself (and, second call, over U): every vector is read before it is written."""
+    g = torch.Generator().manual_seed(77)
+    n, d = 1500, 1024
+    U = (torch.randn(n, d, generator=g) * 0.2).to(torch.bfloat16)
+    H = torch.randn(n, d, generator=g).to(torch.bfloat16)
+    ref_r, ref_Ht = oc.delta_norm(U, H), oc.residual(H, U)
+    for over in ("H", "U"):
+        Ud, Hd = U.to(DEV), H.to(DEV)
+        r = dash.dash_delta_norm(Ud, Hd, Hres_out=Hd if over == "H" else Ud)
+        r_close(r.cpu().numpy(), ref_r)
+        assert_close_rms((Hd if over == "H" else Ud).float().cpu().numpy(), ref_Ht, f"H~ over {over}")
+    # an indexed destination inside an input is refused (a row could be read after another row's result landed on it)
+    with pytest.raises(dash.DashError):
+        dash.dash_delta_norm(U.to(DEV), Hd, Hres_out=Hd, res_index=torch.arange(n, dtype=torch.int32, device=DEV))
+
+
+def test_fold_norm_weight_is_the_once_rounded_product():
+    """W_out[i, j] = w[i] * W[i, j]: the product of two bf16 values is exact in fp32, so the result is that product rounded once."""
+    g = torch.Generator().manual_seed(78)
+    for dtype, d, N in ((torch.bfloat16, 520, 1536), (torch.float32, 64, 100)):
+        W = (torch.randn(d, N, generator=g) * 0.02).to(dtype)
+        w = (1.0 + 0.3 * torch.randn(d, generator=g)).to(dtype)
+        want = torch.from_numpy(oc.f64(w)[:, None] * oc.f64(W)).to(dtype)       # fp64 product, rounded once to the storage type
+        Wd = W.to(DEV)
+        out = dash.dash_fold_norm_weight(Wd, w.to(DEV))
+        assert torch.equal(out.cpu(), want)
+        dash.dash_fold_norm_weight(Wd, w.to(DEV), out=Wd)                        # in place
+        assert torch.equal(Wd.cpu(), want)
+
+
+def test_lookback_wait_gives_up_reports_timeout_and_the_library_carries_on():
+    """Every device-side wait is bounded.  The test hook starts the compaction's tile ticket at 1: tile 0 is never taken and the
+    tile behind it polls a state word that nobody publishes, runs out of polls, reports DASH_ERR_TIMEOUT through the status word
+    and lets the other tiles finish.  The word clears on reading, and the next ordinary call is correct."""
+    cu = wl.cu_from_lengths([40000, 7])
+    n = int(cu[-1])
+    mask = wl.random_mask(n, 0.5, seed=91)
+    out = dash.dash_testing_compact_stalled(mask.to(DEV), cu.to(DEV), spin_limit=1000)
+    torch.cuda.synchronize()                                                      # the kernel returned
+    assert dash.dash_check_status() == 5 and dash.lib().dash_status_string(5) == b"a device-side wait gave up"
+    assert dash.dash_check_status() == dash.OK                                    # reported once, then clear
+    assert 0 <= int(out["n_out"].item()) <= n
+    # an ordinary call of the same size (look-back path) right behind it
+    X = torch.randn(n, 64, generator=torch.Generator().manual_seed(92)).to(torch.bfloat16)
+    got = dash.dash_compact(mask.to(DEV), cu.to(DEV), rows=[X.to(DEV)], pos_in=wl.positions(cu).to(DEV))
+    ref = oc.compact(mask, cu, rows=[X], pos_in=wl.positions(cu))
+    k = ref["n_out"]
+    assert int(got["n_out"].item()) == k and np.array_equal(got["idx"][:k].cpu().numpy(), ref["idx"])
+    assert np.array_equal(got["cu_out"].cpu().numpy(), ref["cu_out"]) and torch.equal(got["rows"][0][:k].cpu(), ref["rows"][0])
+    assert dash.dash_check_status() == dash.OK
+
+
 def test_delta_norm_strided_rows_and_fused_threshold():
     g = torch.Generator().manual_seed(5)
     n, d = 777, 256

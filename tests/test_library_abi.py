@@ -20,12 +20,17 @@ def lib():
     return dash.lib()
 
 
-def test_every_declared_symbol_is_exported(lib):
-    hdr = open(os.path.join(ROOT, "include", "dash.h")).read()
+def _declared(header):
+    hdr = open(os.path.join(ROOT, "include", header)).read()
     hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    declared = set(re.findall(r"\b(dash_[a-z_0-9]+)\s*\(", hdr))
-    assert declared == set(dash.EXPORTS)
-    for name in declared:
+    return set(re.findall(r"\b(dash_[a-z_0-9]+)\s*\(", hdr))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["dash.h", "dash_testing.h"]
+    assert _declared("dash.h") == set(dash.EXPORTS)
+    assert _declared("dash_testing.h") == set(dash.TEST_HOOKS)
+    for name in dash.EXPORTS + dash.TEST_HOOKS:
         assert hasattr(lib, name), name
 
 
@@ -55,8 +60,8 @@ def test_invalid_arguments_are_rejected_before_any_launch(lib):
     # misaligned pointer
     assert lib.dash_delta_norm(ctypes.c_void_p(4100), fake, 4, 16, 16, 16, dash.BF16, 0, 0.0, fake, nul, 0, nul, None, nul, nul) == 1
     # select without sequence boundaries / keep-count without counts
-    assert lib.dash_select(fake, 8, nul, 1, 0, 0.0, nul, 0, 0, fake, nul, 0, nul) == 1
-    assert lib.dash_select(fake, 8, fake, 1, 1, 0.0, nul, 0, 0, fake, nul, 0, nul) == 1
+    assert lib.dash_select(fake, 8, nul, 1, 0, 0.0, nul, 0, 0, fake, nul) == 1
+    assert lib.dash_select(fake, 8, fake, 1, 1, 0.0, nul, 0, 0, fake, nul) == 1
     # compaction: missing / too-small workspace
     assert lib.dash_compact(fake, 8, fake, 1, None, 0, nul, nul, nul, nul, nul, fake, nul, nul, 0, nul) == 3
     assert lib.dash_compact(fake, 1 << 20, fake, 1, None, 0, nul, nul, nul, nul, nul, fake, nul, fake, 512, nul) == 3
