@@ -209,7 +209,7 @@ def setup_block_step(args, dash, dev, rank):
     es = torch.empty(0, dtype=sh.dtype).element_size()
     H_host, pos_host = _pin(w.tensors["H"]), _pin(wl.positions(w.cu))
     tok_host, cu_host = _pin(torch.arange(T, dtype=torch.int32)), _pin(w.cu)
-    layer = dash.Layer(sh, w.weights[0], dev, tau=0.0, fused_projections=not args.library_gemms)
+    layer = dash.Layer(sh, w.weights[0], dev, tau=0.0)
     B = StepBuffers(dash, layer, T, S, sh.d, sh.dtype, dev)
     H = torch.empty(T, sh.d, dtype=sh.dtype, device=dev)
     pos, tok = torch.empty(T, dtype=torch.int32, device=dev), torch.empty(T, dtype=torch.int32, device=dev)
@@ -319,7 +319,7 @@ def setup_cascade(args, dash, dev, rank):
     w = wl.config3(T=T, seed=rank_seed(2, rank), n_layers=Lr)
     sh, S, es = w.shape, w.S, 2
     Ks = [dash.dash_keep_count(T, 1.0 - f) for f in w.fractions]
-    layers = [dash.Layer(sh, w.weights[l], dev, tau=0.0, fused_projections=not args.library_gemms) for l in range(Lr)]
+    layers = [dash.Layer(sh, w.weights[l], dev, tau=0.0) for l in range(Lr)]
     A, Bb = StepBuffers(dash, layers[0], T, S, sh.d, sh.dtype, dev), StepBuffers(dash, layers[0], T, S, sh.d, sh.dtype, dev)
     H_host, pos_host = _pin(w.tensors["H"]), _pin(wl.positions(w.cu))
     tok_host, cu_host = _pin(torch.arange(T, dtype=torch.int32)), _pin(w.cu)
@@ -484,7 +484,7 @@ def setup_stack(args, dash, dev, rank):
     Wt = dict(wl.layer_weights(sh, rank_seed(5, rank))); Wt.update(wl.ffn_weights(sh, rank_seed(5, rank)))
     K = dash.dash_keep_count(T, rho, 64, 32, 1)
     kc = torch.tensor([K], dtype=torch.int32, device=dev)
-    blk = dash.Block(sh, Wt, dev, tau=0.0, keep_first=64, keep_last=32, fused_projections=not args.library_gemms)   # one set of weights (timing only)
+    blk = dash.Block(sh, Wt, dev, tau=0.0, keep_first=64, keep_last=32)   # one set of weights (timing only)
     lay = dash.dash_block_workspace(blk, T, S)
     ws = dash.workspace(lay.total, dev)
     H_host, pos_host = _pin(wl.hidden_states(T, sh.d, rank_seed(5, rank), sh.dtype)), _pin(wl.positions(cu_h))
@@ -749,7 +749,7 @@ def run_ours(args):
     cfg = {"workload": W["workload"], "tokens_per_step_per_gpu": tokens,
            "l2": f"flushed between timed steps ({L2_FLUSH_BYTES >> 20} MiB write, then {L2_FLUSH_BYTES >> 20} MiB read)", "status_word": status}
     cfg.update(W["extra"])
-    cfg["projections"] = "library GEMMs (cuBLASLt)" if args.library_gemms else "this library's tcgen05 GEMMs (CTA pairs) with fused epilogues"
+    cfg["projections"] = "this library's tcgen05 GEMMs (CTA pairs) with fused epilogues"
     out = {
         "metric": METRIC, "value": whole_job_value(tokens, world, t_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": t_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -926,8 +926,6 @@ def main():
     ap.add_argument("--indexed-attention", action="store_true",
                     help="cfg4 / cfg5: leave Q full-length and fetch its active rows by index in the attention kernel (dash_varlen_attention_indexed) "
                          "instead of compacting Q")
-    ap.add_argument("--library-gemms", action="store_true",
-                    help="block steps use the library GEMMs (cuBLASLt) for the projections instead of this library's tcgen05 GEMMs with fused epilogues")
     args = ap.parse_args()
     if args.seq is None:
         args.seq = {"cfg1": 1024, "cfg2": 8192, "cfg3": 32768}.get(args.workload, 8192)

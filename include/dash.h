@@ -251,16 +251,19 @@ typedef struct {
     int          scatter_which;    /* rows of H~ written to x_full: 0 halted, 2 all */
     void*        k_cache;          /* NULL, or [n, Hkv, D]: this block's keys (rotary applied) of the entering tokens, */
     void*        v_cache;          /* and values: the rows a decoding step attends over at this depth (both or neither) */
-    int          fused_projections; /* 1 (what the binding sets by default): the projections run in this library's tcgen05 GEMMs
-                                     * (256 x 256 tiles on CTA pairs) with the work that follows them on the accumulators: rotary
-                                     * embedding in the QKV projection; H~ and the score's row sums in the output projection;
-                                     * SwiGLU in the gate | up projection -- one rounding less per value, no U and no gate | up
-                                     * intermediate.  bf16 with 256-column tiles; other shapes and fp32 fall back to 0.
-                                     * 0: library GEMMs (cuBLASLt), rotary embedding, residual and score in passes of this library. */
-    int          rms_folded;       /* 1: the norm's weight is already in Wqkv (row i of Wqkv multiplied by rms_weight[i]; rms_weight
-                                    * may then be NULL): the norm costs no pass of its own -- one pass over H yields the row factors
-                                    * 1 / rms, which the projection applies to its accumulators.  Needs fused_projections. */
+    int          rms_folded;       /* 1: the norm's weight is already in Wqkv (dash_fold_norm_weight; rms_weight may then be NULL):
+                                    * the norm costs no pass of its own -- one pass over H yields the row factors 1 / rms, which
+                                    * the projection applies to its accumulators.  Only where the projections run with their
+                                    * fused epilogues (see below); DASH_ERR_UNSUPPORTED otherwise. */
 } dash_layer_cfg;
+/* The projections (Wqkv, Wo; Wgu, Wd of dash_block_step) run in this library's tcgen05 GEMMs (256 x 256 tiles on CTA pairs).
+ * bf16 tensors whose projections have whole 256-column tiles ((Hq + 2 Hkv) D, (Hq + Hkv) D and d multiples of 256, d and Hq D
+ * multiples of 64; the FFN width a multiple of 128) get the work that follows a projection on its accumulators: the rotary
+ * embedding in the QKV projection; H~ and the score's row sums in the output projection; SwiGLU in the gate | up projection --
+ * one rounding less per value, no U and no gate | up intermediate.  Other shapes (rows must still start on 16-byte boundaries:
+ * d, Hq D, m multiples of 8) and fp32 tensors run the same GEMM kernel plain, with the norm, the rotary embedding, the residual
+ * and the score as passes of their own; fp32 operands are rounded to bf16 copies in the workspace first (fp32 accumulation,
+ * fp32 results), as the attention kernel does with Q, K, V. */
 
 /* LN of Eq. 1 is read as RMSNorm, y = x / rms(x) * w.  Its weight w can be folded, once and ahead of time, into the
  * projection that follows the norm: W_out[i, j] = w[i] * W[i, j] for W, W_out [d, N] row-major of type dt (row strides ldw,
@@ -300,8 +303,7 @@ int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, const int32_t* 
  * come from U.  FFN is the gated feed-forward of the Qwen2.5 backbones:
  * FFN(x) = (silu(x Wg) * (x Wu)) Wd.  H' of every entering token is written to x_full
  * (attn.scatter_which must be 2: H' is also the last updated value of the tokens that
- * halt here, Sec. 3.4), H' of the tokens that stay to H_next.  Projections are library
- * GEMMs; everything else runs in this library's kernels. */
+ * halt here, Sec. 3.4), H' of the tokens that stay to H_next. */
 typedef struct {
     dash_layer_cfg attn;
     int          m;                /* feed-forward width, multiple of 8 */
@@ -309,7 +311,7 @@ typedef struct {
     const void*  Wd;               /* [m, d] */
     const void*  rms2_weight;      /* [d]: weight of the norm in front of the FFN (attn.rms_eps is used) */
     dash_signal  signal;           /* what the score measures */
-    int          rms2_folded;      /* as attn.rms_folded, for the norm in front of the FFN and Wgu (needs DASH_SIGNAL_ATTN) */
+    int          rms2_folded;      /* as attn.rms_folded, for the norm in front of the FFN and Wgu (needs DASH_SIGNAL_ATTN and attn.rms_folded) */
 } dash_block_cfg;
 typedef struct {
     dash_layer_ws_layout attn;

@@ -520,6 +520,14 @@ __global__ void f32_to_bf16_rows_kernel(const float* __restrict__ src, int64_t l
     }
 }
 
+int launch_f32_to_bf16(const float* src, int64_t ld_src, void* dst, int64_t ld_dst, int64_t rows, int64_t cols, cudaStream_t st) {
+    if (rows <= 0 || cols <= 0) return DASH_OK;
+    int64_t grid = (rows * (cols / 4) + 255) / 256, cap = (int64_t)sm_count() * 8;
+    if (grid > cap) grid = cap;
+    f32_to_bf16_rows_kernel<<<(int)grid, 256, 0, st>>>(src, ld_src, (__nv_bfloat16*)dst, ld_dst, rows, (int)cols);
+    return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
+}
+
 // workspace: [0,256) ticket + item count; then the plan (one int4 per existing (sequence, query tile));
 // then, for fp32 tensors, their bf16 copies
 static size_t plan_entries(int64_t n, int S) { return (size_t)(n / kBM) + (size_t)S + 1; }

@@ -1,6 +1,9 @@
 // Projections of the block as persistent tcgen05 GEMMs: C[n, N] = A[n, K] W[K, N], bf16 operands, fp32 accumulation in
 // TMEM, with the element-wise work that follows each projection done on the accumulators before anything is written:
-//   PLAIN  : C = A W                                                   (down projection of the FFN)
+//   PLAIN  : C = A W (bf16 or fp32 out; any N, K that keep rows 16-byte aligned: tiles past the edge of W or along K are
+//            zero-filled by the loads, columns past N are not stored)   (down projection of the FFN; every projection of the
+//            path that runs the norm, the rotary embedding and the residual as passes of their own; fp32 tensors, whose
+//            operands are rounded to bf16 copies first)
 //   ROPE   : Q | K | V = Hn Wqkv with the rotary embedding applied to the Q and K heads    (Eq. 1, inside Attn)
 //   RESID  : U = O Wo is never stored: H~ = H + U goes straight to x_full[tok[row]], and the per-row partial sums of
 //            u^2, h^2 and (h+u)^2 of this tile's columns go to a small buffer (the score of Eq. 2 and the next norm's row factor are
@@ -77,6 +80,7 @@ struct GemmArgs {
     int n, N, K;                 // rows (upper bound), columns of W that one tile row of the output spans, depth
     int n_tiles;                 // tiles along the output columns
     void* C; int64_t ldc;        // PLAIN / ROPE / SWIGLU output (elements)
+    int out_f32;                 // PLAIN: C is fp32 (else bf16)
     const int32_t* n_dev;        // device: true number of rows (<= n), or null
     int* status;
     GemmEpilogue e;
@@ -117,7 +121,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     cluster_sync_all();                                    // the peer's barriers exist before anything is signalled across
     tc_fence_after();
     const uint32_t tmem = *slot_gen;
-    const int m_tiles = (g.n + 2 * kGM - 1) / (2 * kGM), n_tiles = g.n_tiles, tiles = m_tiles * n_tiles, ksteps = g.K / kGK;
+    const int m_tiles = (g.n + 2 * kGM - 1) / (2 * kGM), n_tiles = g.n_tiles, tiles = m_tiles * n_tiles, ksteps = (g.K + kGK - 1) / kGK;
     const int n_pairs = (int)gridDim.x / 2, pair = (int)blockIdx.x / 2;
     constexpr uint32_t idesc = idesc_bf16_f32(2 * kGM, kGN, false, true);
     constexpr uint32_t hi = smem_desc_hi_sw128(1024);
@@ -194,19 +198,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             const bool live = row < n_true;
             const uint32_t tD = tmem + b * kGN + lane_base;
             if (EPI == GEMM_PLAIN) {
-                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.C) + (int64_t)row * g.ldc + nt * kGN;
+                // columns at or past N (a last, partial tile) are not stored; N is a multiple of 8 (bf16) / 4 (fp32)
+                const int col0 = nt * kGN;
 #pragma unroll
                 for (int c = 0; c < kGN / 32; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tD + c * 32, o);
                     tmem_wait_ld();
-                    if (live) {
+                    if (live && g.out_f32) {
+                        float* dst = reinterpret_cast<float*>(g.C) + (int64_t)row * g.ldc + col0 + c * 32;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            if (col0 + c * 32 + e < g.N) st_v4(dst + e, make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]));
+                    } else if (live) {
+                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.C) + (int64_t)row * g.ldc + col0 + c * 32;
 #pragma unroll
                         for (int e = 0; e < 32; e += 8)
-                            st_v4(dst + c * 32 + e, make_uint4(pack_bf16(__uint_as_float(o[e]), __uint_as_float(o[e + 1])),
-                                                               pack_bf16(__uint_as_float(o[e + 2]), __uint_as_float(o[e + 3])),
-                                                               pack_bf16(__uint_as_float(o[e + 4]), __uint_as_float(o[e + 5])),
-                                                               pack_bf16(__uint_as_float(o[e + 6]), __uint_as_float(o[e + 7]))));
+                            if (col0 + c * 32 + e < g.N)
+                                st_v4(dst + e, make_uint4(pack_bf16(__uint_as_float(o[e]), __uint_as_float(o[e + 1])),
+                                                          pack_bf16(__uint_as_float(o[e + 2]), __uint_as_float(o[e + 3])),
+                                                          pack_bf16(__uint_as_float(o[e + 4]), __uint_as_float(o[e + 5])),
+                                                          pack_bf16(__uint_as_float(o[e + 6]), __uint_as_float(o[e + 7]))));
                     }
                 }
             } else if (EPI == GEMM_ROPE) {
@@ -381,7 +393,10 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mw, const GemmA
 }
 
 bool gemm_shape_ok(GemmEpilogueKind kind, int64_t n, int64_t N, int64_t K, int64_t lda, int64_t ldw, const GemmEpilogue& e) {
-    if (n < 1 || n > 0x7fffffffLL || K < kGK || (K % kGK) || (lda % 8) || (ldw % 8)) return false;
+    if (n < 1 || n > 0x7fffffffLL || N < 1 || N > 0x7fffffffLL || K < 1 || K > 0x7fffffffLL || (lda % 8) || (ldw % 8)) return false;
+    if (kind == GEMM_PLAIN) return (N % 4) == 0 && (K % 8) == 0;      // rows of A, W and C start on 16-byte boundaries
+    // the fused epilogues work on whole 256-column tiles and whole K steps
+    if (K < kGK || (K % kGK)) return false;
     if (kind == GEMM_SWIGLU) return e.m >= 128 && (e.m % 128) == 0 && N == 2 * (int64_t)e.m;
     if (N < kGN || (N % kGN)) return false;
     if (kind == GEMM_ROPE) return (e.D == 64 || e.D == 128) && (e.n_rot_cols % kGN) == 0 && e.n_rot_cols <= N;
@@ -389,17 +404,19 @@ bool gemm_shape_ok(GemmEpilogueKind kind, int64_t n, int64_t N, int64_t K, int64
 }
 
 int gemm_bf16(GemmEpilogueKind kind, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc, int64_t n, int64_t N,
-              int64_t K, const GemmEpilogue& e, const int32_t* n_dev, cudaStream_t st) {
+              int64_t K, const GemmEpilogue& e, const int32_t* n_dev, cudaStream_t st, bool out_f32) {
     if (!gemm_shape_ok(kind, n, N, K, lda, ldw, e)) return DASH_ERR_UNSUPPORTED;
     if (!aligned16(A) || !aligned16(W)) return DASH_ERR_INVALID_ARG;
+    if (out_f32 && kind != GEMM_PLAIN) return DASH_ERR_UNSUPPORTED;
+    if (kind == GEMM_PLAIN && (!aligned16(C) || (ldc * (out_f32 ? 4 : 2)) % 16 || (!out_f32 && (N % 8)))) return DASH_ERR_UNSUPPORTED;
     CUtensorMap ma, mw;
     int rc;
     if ((rc = make_map_2d_bf16(&ma, A, (uint64_t)K, (uint64_t)n, (uint64_t)lda, 64, kGM)) != DASH_OK) return rc;
     if ((rc = make_map_2d_bf16(&mw, W, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, 64, kGK)) != DASH_OK) return rc;
     GemmArgs g;
     g.n = (int)n; g.N = (int)N; g.K = (int)K;
-    g.n_tiles = kind == GEMM_SWIGLU ? e.m / 128 : (int)(N / kGN);
-    g.C = C; g.ldc = ldc; g.n_dev = n_dev; g.e = e;
+    g.n_tiles = kind == GEMM_SWIGLU ? e.m / 128 : (int)((N + kGN - 1) / kGN);
+    g.C = C; g.ldc = ldc; g.n_dev = n_dev; g.e = e; g.out_f32 = out_f32 ? 1 : 0;
     g.status = status_word_ptr();
     if (!g.status) return DASH_ERR_CUDA;
     switch (kind) {

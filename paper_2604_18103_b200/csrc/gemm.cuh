@@ -27,11 +27,16 @@ struct GemmEpilogue {
     int m = 0;
 };
 
-// true if the own kernel takes this problem (bf16, 256-column tiles, K in steps of 64); otherwise the caller uses the library GEMM
+// true if the kernel takes this problem with this epilogue.  PLAIN: any N % 4 == 0, K % 8 == 0 (rows on 16-byte boundaries); the
+// fused epilogues: whole 256-column tiles (SWIGLU: m % 128 == 0) and K in steps of 64 -- otherwise the caller runs the projection
+// PLAIN and the element-wise work as passes of their own.
 bool gemm_shape_ok(GemmEpilogueKind kind, int64_t n, int64_t N, int64_t K, int64_t lda, int64_t ldw, const GemmEpilogue& e);
-// C (or the epilogue's outputs) = A[n, K] W[K, N]; ld* in elements; n_dev: device true row count or null
+// C (or the epilogue's outputs) = A[n, K] W[K, N], A and W bf16; ld* in elements; n_dev: device true row count or null;
+// out_f32 (PLAIN only): C is fp32 instead of bf16
 int gemm_bf16(GemmEpilogueKind kind, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc, int64_t n, int64_t N,
-              int64_t K, const GemmEpilogue& e, const int32_t* n_dev, cudaStream_t st);
+              int64_t K, const GemmEpilogue& e, const int32_t* n_dev, cudaStream_t st, bool out_f32 = false);
+// dst (bf16, row stride ld_dst) = src (fp32, row stride ld_src) rounded to nearest even; cols % 4 == 0
+int launch_f32_to_bf16(const float* src, int64_t ld_src, void* dst, int64_t ld_dst, int64_t rows, int64_t cols, cudaStream_t st);
 // per row: (cos, sin) of pos * base^(-2i/D) into table [n, D/2]; with inv_rms non-null also 1 / sqrt(mean(H_row^2) + eps) (bf16 H, row stride ldh)
 int launch_row_prep(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const void* H, int64_t ldh, int d, float rms_eps,
                     float* inv_rms, const int32_t* n_dev, cudaStream_t st);

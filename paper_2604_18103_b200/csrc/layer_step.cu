@@ -2,14 +2,10 @@
 // on the packed active tokens: RMSNorm -> QKV projection -> rotary embedding ->
 // causal attention -> output projection -> delta score / residual / halting rule
 // -> scatter of the updated states -> compaction of the tokens that stay active.
-// The two projections are plain library GEMMs (cuBLASLt); everything else runs in
-// this library's own kernels.  One stream, no host synchronisation.
-#include <cublasLt.h>
+// Every step runs in this library's own kernels; the projections are the tcgen05 GEMMs of gemm.cu -- with the norm's row
+// factor, the rotary embedding, the residual and the score's row sums on their accumulators where the shapes allow it (bf16,
+// whole 256-column tiles), as plain GEMMs between passes of their own otherwise.  One stream, no host synchronisation.
 #include <math.h>
-
-#include <map>
-#include <mutex>
-#include <tuple>
 
 #include "common.cuh"
 #include "gemm.cuh"
@@ -115,57 +111,6 @@ rope_kernel(char* __restrict__ X, int64_t ldx_b, const int32_t* __restrict__ pos
     }
 }
 
-// ---- library GEMM: C[n, N] = A[n, K] * W[K, N], all row-major ---------------------
-struct LtState {
-    cublasLtHandle_t handle = nullptr;
-    std::mutex mu;
-    std::map<std::tuple<int, int64_t, int64_t, int64_t, int64_t, int64_t, int64_t>, cublasLtMatmulAlgo_t> algos;
-};
-static LtState& lt() { static LtState s; return s; }
-constexpr size_t kLtWorkspace = 64ull << 20;
-
-static int gemm_rowmajor(dash_dtype dt, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc,
-                         int64_t n, int64_t N, int64_t K, void* lt_ws, cudaStream_t st) {
-    LtState& s = lt();
-    std::lock_guard<std::mutex> g(s.mu);
-    if (!s.handle && cublasLtCreate(&s.handle) != CUBLAS_STATUS_SUCCESS) return DASH_ERR_CUDA;
-    const cudaDataType_t ty = (dt == DASH_BF16) ? CUDA_R_16BF : CUDA_R_32F;
-    cublasLtMatmulDesc_t op = nullptr;
-    cublasLtMatrixLayout_t la = nullptr, lb = nullptr, lc = nullptr;
-    int rc = DASH_ERR_CUDA;
-    const float alpha = 1.f, beta = 0.f;
-    do {
-        if (cublasLtMatmulDescCreate(&op, CUBLAS_COMPUTE_32F, CUDA_R_32F) != CUBLAS_STATUS_SUCCESS) break;
-        // row-major C = A W  <=>  column-major C^T[N,n] = W^T[N,K] A^T[K,n]
-        if (cublasLtMatrixLayoutCreate(&la, ty, N, K, ldw) != CUBLAS_STATUS_SUCCESS) break;
-        if (cublasLtMatrixLayoutCreate(&lb, ty, K, n, lda) != CUBLAS_STATUS_SUCCESS) break;
-        if (cublasLtMatrixLayoutCreate(&lc, ty, N, n, ldc) != CUBLAS_STATUS_SUCCESS) break;
-        auto key = std::make_tuple((int)dt, n, N, K, lda, ldw, ldc);
-        auto it = s.algos.find(key);
-        if (it == s.algos.end()) {
-            cublasLtMatmulPreference_t pref = nullptr;
-            if (cublasLtMatmulPreferenceCreate(&pref) != CUBLAS_STATUS_SUCCESS) break;
-            size_t wsz = kLtWorkspace;
-            cublasLtMatmulPreferenceSetAttribute(pref, CUBLASLT_MATMUL_PREF_MAX_WORKSPACE_BYTES, &wsz, sizeof(wsz));
-            cublasLtMatmulHeuristicResult_t res;
-            int found = 0;
-            cublasStatus_t hs = cublasLtMatmulAlgoGetHeuristic(s.handle, op, la, lb, lc, lc, pref, 1, &res, &found);
-            cublasLtMatmulPreferenceDestroy(pref);
-            if (hs != CUBLAS_STATUS_SUCCESS || found < 1) break;
-            it = s.algos.emplace(key, res.algo).first;
-        }
-        if (cublasLtMatmul(s.handle, op, &alpha, W, la, A, lb, &beta, C, lc, C, lc, &it->second, lt_ws, kLtWorkspace, st) !=
-            CUBLAS_STATUS_SUCCESS)
-            break;
-        rc = DASH_OK;
-    } while (0);
-    if (la) cublasLtMatrixLayoutDestroy(la);
-    if (lb) cublasLtMatrixLayoutDestroy(lb);
-    if (lc) cublasLtMatrixLayoutDestroy(lc);
-    if (op) cublasLtMatmulDescDestroy(op);
-    return rc;
-}
-
 int launch_sums_to_score(const float4* sums, int n_sum_tiles, int64_t n, dash_norm_mode mode, float eps, float* r_out, const dash_threshold* fused,
                          const int32_t* n_dev, float* inv_rms_out, int d, float rms_eps, cudaStream_t st);
 int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float4* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
@@ -178,13 +123,24 @@ int attention_planned(const void* Q, const void* K, const void* V, void* O, floa
                       const int32_t* cu_seqlens, int S, int64_t n, int64_t max_seqlen, int Hq, int Hkv, int D, float scale, dash_dtype dt,
                       void* ws, size_t ws_bytes, cudaStream_t st);
 
-// C = A W: this library's GEMM when it takes the problem (bf16, 256-column tiles), the library GEMM otherwise
-static int project(bool own, dash_dtype dt, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc, int64_t n, int64_t N, int64_t K,
-                   const int32_t* n_dev, void* lt_ws, cudaStream_t st) {
+// Room for the bf16 copies of the operands of a projection on fp32 tensors
+struct ConvScratch { char* a; size_t a_bytes; char* w; size_t w_bytes; };
+static size_t conv_a_bytes(int64_t n, int64_t k_max) { return align_up((size_t)n * align_up((size_t)k_max, 8) * 2, 256); }
+static size_t conv_w_bytes(int64_t k, int64_t n_cols) { return align_up((size_t)k * align_up((size_t)n_cols, 8) * 2, 256); }
+
+// C = A W (plain).  bf16: the GEMM of gemm.cu as it is.  fp32: its operands are rounded to bf16 copies first (what the
+// attention kernel does with Q, K, V), the product accumulates in fp32 and is stored as fp32.
+static int project(dash_dtype dt, const void* A, int64_t lda, const void* W, int64_t ldw, void* C, int64_t ldc, int64_t n, int64_t N, int64_t K,
+                   const int32_t* n_dev, const ConvScratch& cs, cudaStream_t st) {
     GemmEpilogue e;
-    if (own && dt == DASH_BF16 && gemm_shape_ok(GEMM_PLAIN, n, N, K, lda, ldw, e) && aligned16(C) && (ldc % 8) == 0)
-        return gemm_bf16(GEMM_PLAIN, A, lda, W, ldw, C, ldc, n, N, K, e, n_dev, st);
-    return gemm_rowmajor(dt, A, lda, W, ldw, C, ldc, n, N, K, lt_ws, st);
+    if (dt == DASH_BF16) return gemm_bf16(GEMM_PLAIN, A, lda, W, ldw, C, ldc, n, N, K, e, n_dev, st);
+    if ((K % 8) || (N % 4)) return DASH_ERR_UNSUPPORTED;
+    const int64_t lda_b = K, ldw_b = (int64_t)align_up((size_t)N, 8);
+    if ((size_t)n * lda_b * 2 > cs.a_bytes || (size_t)K * ldw_b * 2 > cs.w_bytes) return DASH_ERR_WORKSPACE;
+    int rc;
+    if ((rc = launch_f32_to_bf16((const float*)A, lda, cs.a, lda_b, n, K, st)) != DASH_OK) return rc;
+    if ((rc = launch_f32_to_bf16((const float*)W, ldw, cs.w, ldw_b, K, N, st)) != DASH_OK) return rc;
+    return gemm_bf16(GEMM_PLAIN, cs.a, lda_b, cs.w, ldw_b, C, ldc, n, N, K, e, n_dev, st, true);
 }
 
 static int rows_grid8(int64_t n) {
@@ -259,7 +215,6 @@ static bool cfg_ok(const dash_layer_cfg* c) {
     if (c->scatter_which != 0 && c->scatter_which != 2) return false;
     if (!(c->rope_base > 0.0)) return false;
     if ((c->k_cache == nullptr) != (c->v_cache == nullptr)) return false;
-    if (c->fused_projections != 0 && c->fused_projections != 1) return false;
     return true;
 }
 
@@ -294,8 +249,12 @@ extern "C" int dash_layer_workspace(const dash_layer_cfg* cfg, int64_t n, int S,
     out->O = off;   off += align_up((size_t)n * cfg->Hq * cfg->D * es, 256);
     out->U = off;   off += align_up((size_t)n * cfg->d * es, 256);
     out->Ht = off;  off += align_up((size_t)n * cfg->d * es, 256);
-    out->scratch = off;
-    off += kLtWorkspace;
+    out->scratch = off;                    // fp32 tensors: bf16 copies of a projection's operands (activations, then weights)
+    if (cfg->dt == DASH_F32) {
+        const int64_t hd = (int64_t)cfg->Hq * cfg->D;
+        off += conv_a_bytes(n, cfg->d > hd ? cfg->d : hd);
+        off += conv_w_bytes(cfg->d, (int64_t)nq > cfg->d ? (int64_t)nq : cfg->d) > conv_w_bytes(hd, cfg->d) ? conv_w_bytes(cfg->d, (int64_t)nq > cfg->d ? (int64_t)nq : cfg->d) : conv_w_bytes(hd, cfg->d);
+    }
     off += align_up(dash_workspace_bytes(DASH_WS_COMPACT, n, S, 0, 0, 0, cfg->dt), 256);
     off += align_up(dash_workspace_bytes(DASH_WS_ATTENTION, n, S, cfg->Hq, cfg->Hkv, cfg->D, cfg->dt), 256);
     off += align_up((size_t)n * (cfg->D / 2) * sizeof(float2), 256);              // (cos, sin) of every row for the QKV epilogue
@@ -309,7 +268,8 @@ namespace dash {
 
 struct StepWs {
     dash_layer_ws_layout L;
-    char *Hn, *QKV, *O, *U, *Ht, *lt_ws, *compact_ws, *attn_ws;
+    char *Hn, *QKV, *O, *U, *Ht, *compact_ws, *attn_ws;
+    ConvScratch conv;
     size_t compact_bytes, attn_bytes;
     float2* rope_tab;
     float4* sums;
@@ -321,8 +281,17 @@ static int carve_ws(const dash_layer_cfg* cfg, int64_t n, int S, void* ws, StepW
     if (rc != DASH_OK) return rc;
     char* w = (char*)ws;
     out->Hn = w + out->L.Hn; out->QKV = w + out->L.QKV; out->O = w + out->L.O; out->U = w + out->L.U; out->Ht = w + out->L.Ht;
-    out->lt_ws = w + out->L.scratch;
-    out->compact_ws = out->lt_ws + kLtWorkspace;
+    out->conv = {nullptr, 0, nullptr, 0};
+    char* after = w + out->L.scratch;
+    if (cfg->dt == DASH_F32) {
+        const int64_t hd = (int64_t)cfg->Hq * cfg->D, nq = (int64_t)(cfg->Hq + 2 * cfg->Hkv) * cfg->D;
+        const size_t ab = conv_a_bytes(n, cfg->d > hd ? cfg->d : hd);
+        const size_t w1 = conv_w_bytes(cfg->d, nq > cfg->d ? nq : cfg->d), w2 = conv_w_bytes(hd, cfg->d);
+        const size_t wb = w1 > w2 ? w1 : w2;
+        out->conv = {after, ab, after + ab, wb};
+        after += ab + wb;
+    }
+    out->compact_ws = after;
     out->compact_bytes = align_up(dash_workspace_bytes(DASH_WS_COMPACT, n, S, 0, 0, 0, cfg->dt), 256);
     out->attn_ws = out->compact_ws + out->compact_bytes;
     out->attn_bytes = dash_workspace_bytes(DASH_WS_ATTENTION, n, S, cfg->Hq, cfg->Hkv, cfg->D, cfg->dt);
@@ -357,7 +326,7 @@ static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int
     if ((rc = attention_plan(cu_in, S, n, Hq, W.attn_ws, W.attn_bytes, st)) != DASH_OK) return rc;
     GemmEpilogue e;
     e.D = D; e.n_rot_cols = (Hq + Hkv) * D; e.rope_table = W.rope_tab;
-    const bool fused = bf && cfg->fused_projections && gemm_shape_ok(GEMM_ROPE, n, nq, d, d, nq, e);
+    const bool fused = bf && gemm_shape_ok(GEMM_ROPE, n, nq, d, d, nq, e);
     if (fused && cfg->rms_folded) {
         // LN folded into the projection: its weight sits in Wqkv, its row factor 1 / rms is applied to the accumulators.
         // One pass over H gives the row factors and the rotary angles; Q | K | V = (H Wqkv) / rms, Q and K rotated.
@@ -372,7 +341,7 @@ static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int
     } else {
         if (cfg->rms_folded) return DASH_ERR_UNSUPPORTED;      // folded weights need the fused projection (bf16, 256-column tiles)
         if ((rc = launch_rmsnorm(cfg->dt, H_in, cfg->rms_weight, W.Hn, n, d, cfg->rms_eps, n_dev, st)) != DASH_OK) return rc;
-        if ((rc = project(cfg->fused_projections != 0, cfg->dt, W.Hn, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, n_dev, W.lt_ws, st)) != DASH_OK) return rc;
+        if ((rc = project(cfg->dt, W.Hn, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, n_dev, W.conv, st)) != DASH_OK) return rc;
         // rotary embedding on the Q and K heads
         RopeFreq fr;
         for (int i = 0; i < D / 2; ++i) fr.inv_freq[i] = pow(cfg->rope_base, -2.0 * i / D);
@@ -398,7 +367,7 @@ static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int
 // U = O Wo  (pre-residual attention output, Eq. 1) into W.U
 static int out_proj_U(const dash_layer_cfg* cfg, const int32_t* cu_in, int S, int64_t n, const StepWs& W, cudaStream_t st) {
     const int64_t hd = (int64_t)cfg->Hq * cfg->D;
-    return project(cfg->fused_projections != 0, cfg->dt, W.O, hd, cfg->Wo, cfg->d, W.U, cfg->d, n, cfg->d, hd, cu_in + S, W.lt_ws, st);
+    return project(cfg->dt, W.O, hd, cfg->Wo, cfg->d, W.U, cfg->d, n, cfg->d, hd, cu_in + S, W.conv, st);
 }
 
 // Output projection with the residual in its epilogue: dst[idx[row]] = H + O Wo (idx null: row), per-row sums of u^2, h^2 into W.sums.
@@ -408,7 +377,7 @@ static int out_proj_residual(const dash_layer_cfg* cfg, const void* H_in, const 
     const int64_t hd = (int64_t)cfg->Hq * cfg->D;
     GemmEpilogue e;
     e.H = H_in; e.ldh = cfg->d; e.tok_index = idx; e.x_full = dst; e.ldx = cfg->d; e.sums = W.sums;
-    if (!cfg->fused_projections || cfg->dt != DASH_BF16 || !gemm_shape_ok(GEMM_RESID, n, cfg->d, hd, hd, cfg->d, e)) return DASH_ERR_UNSUPPORTED;
+    if (cfg->dt != DASH_BF16 || !gemm_shape_ok(GEMM_RESID, n, cfg->d, hd, hd, cfg->d, e)) return DASH_ERR_UNSUPPORTED;
     return gemm_bf16(GEMM_RESID, W.O, hd, cfg->Wo, cfg->d, nullptr, 0, n, cfg->d, hd, e, cu_in + S, st);
 }
 
@@ -470,7 +439,7 @@ extern "C" int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, cons
                                          cfg->keep_first, cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out,
                                          tok_index_next, pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, true, st);
             if (rc != DASH_ERR_UNSUPPORTED) return rc;
-            // shapes this library's GEMM does not take: U through the library GEMM, then r, H~, the rule, scatter and compaction in one pass
+            // fp32, or shapes without whole 256-column tiles: U through the plain GEMM, then r, H~, the rule, scatter and compaction in one pass
             if ((rc = out_proj_U(cfg, cu_in, S, n, W, st)) != DASH_OK) return rc;
             return launch_delta_tail(W.U, H_in, nullptr, nullptr, 0, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau, cfg->keep_first,
                                      cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out, tok_index_next,
@@ -497,6 +466,10 @@ extern "C" int dash_block_workspace(const dash_block_cfg* cfg, int64_t n, int S,
     out->GU = off;  off += align_up((size_t)n * 2 * cfg->m * es, 256);
     out->ACT = off; off += align_up((size_t)n * cfg->m * es, 256);
     out->F = off;   off += align_up((size_t)n * cfg->attn.d * es, 256);
+    if (cfg->attn.dt == DASH_F32) {        // bf16 copies of the operands of the feed-forward's projections
+        off += conv_a_bytes(n, cfg->m > cfg->attn.d ? cfg->m : cfg->attn.d);
+        off += conv_w_bytes(cfg->attn.d, 2 * (int64_t)cfg->m) > conv_w_bytes(cfg->m, cfg->attn.d) ? conv_w_bytes(cfg->attn.d, 2 * (int64_t)cfg->m) : conv_w_bytes(cfg->m, cfg->attn.d);
+    }
     out->total = off;
     return DASH_OK;
 }
@@ -521,6 +494,13 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
     const int es = a->dt == DASH_BF16 ? 2 : 4;
     const int d = a->d, m = cfg->m;
     char *GU = (char*)ws + BL.GU, *ACT = (char*)ws + BL.ACT, *F = (char*)ws + BL.F;
+    ConvScratch conv = {nullptr, 0, nullptr, 0};
+    if (a->dt == DASH_F32) {
+        char* c0 = F + align_up((size_t)n * d * es, 256);
+        const size_t ab = conv_a_bytes(n, m > d ? m : d);
+        const size_t w1 = conv_w_bytes(d, 2 * (int64_t)m), w2 = conv_w_bytes(m, d);
+        conv = {c0, ab, c0 + ab, w1 > w2 ? w1 : w2};
+    }
     if (n == 0) {
         return dash_compact(mask_out, 0, cu_in, S, nullptr, 0, pos_in, pos_next, tok_index_in, tok_index_next, nullptr, cu_next, n_next_dev,
                             W.compact_ws, W.compact_bytes, st);
@@ -553,7 +533,7 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
     // F = FFN(LN(H~)): gate | up projection, silu(gate) * up, down projection
     GemmEpilogue eg;
     eg.m = m;
-    const bool fused_ffn = a->fused_projections && a->dt == DASH_BF16 && gemm_shape_ok(GEMM_SWIGLU, n, 2 * (int64_t)m, d, d, 2 * (int64_t)m, eg);
+    const bool fused_ffn = a->dt == DASH_BF16 && gemm_shape_ok(GEMM_SWIGLU, n, 2 * (int64_t)m, d, d, 2 * (int64_t)m, eg);
     if (cfg->rms2_folded && !(fused_ffn && have_inv_rms2)) return DASH_ERR_UNSUPPORTED;   // folded weights need the fused projections
     if (!cfg->rms2_folded && (rc = launch_rmsnorm(a->dt, W.Ht, cfg->rms2_weight, W.Hn, n, d, a->rms_eps, n_dev, st)) != DASH_OK) return rc;
     if (fused_ffn) {
@@ -562,7 +542,7 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         eg.row_scale = cfg->rms2_folded ? W.inv_rms2 : nullptr;
         if ((rc = gemm_bf16(GEMM_SWIGLU, cfg->rms2_folded ? W.Ht : W.Hn, d, cfg->Wgu, 2 * (int64_t)m, ACT, m, n, 2 * (int64_t)m, d, eg, n_dev, st)) != DASH_OK) return rc;
     } else {
-        if ((rc = gemm_rowmajor(a->dt, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, GU, 2 * (int64_t)m, n, 2 * (int64_t)m, d, W.lt_ws, st)) != DASH_OK) return rc;
+        if ((rc = project(a->dt, W.Hn, d, cfg->Wgu, 2 * (int64_t)m, GU, 2 * (int64_t)m, n, 2 * (int64_t)m, d, n_dev, conv, st)) != DASH_OK) return rc;
         const int64_t total = n * (int64_t)(m / (16 / es));
         int64_t blocks = (total + 255) / 256, cap = (int64_t)sm_count() * 16;
         if (blocks > cap) blocks = cap;
@@ -570,7 +550,7 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
         else swiglu_kernel<false><<<(int)blocks, 256, 0, st>>>(GU, 2 * (int64_t)m * es, ACT, (int64_t)m * es, n, m, n_dev);
         DASH_CUDA_TRY(cudaGetLastError());
     }
-    if ((rc = project(a->fused_projections != 0, a->dt, ACT, m, cfg->Wd, d, F, d, n, d, m, n_dev, W.lt_ws, st)) != DASH_OK) return rc;
+    if ((rc = project(a->dt, ACT, m, cfg->Wd, d, F, d, n, d, m, n_dev, conv, st)) != DASH_OK) return rc;
     if (cfg->signal == DASH_SIGNAL_BLOCK) {
         // ablation: score = change over the whole block, H' - H = U + F (formed in the gate | up buffer, free by now)
         if ((rc = dash_delta_norm(F, W.U, n, d, d, d, a->dt, DASH_NORM_ABS, a->norm_eps, r_out, GU, d, nullptr, nullptr, n_dev, st)) != DASH_OK) return rc;

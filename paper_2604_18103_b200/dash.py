@@ -52,7 +52,7 @@ class LayerCfg(Structure):
                 ("Wqkv", c_void_p), ("Wo", c_void_p), ("rms_weight", c_void_p), ("rms_eps", c_float),
                 ("rope_base", c_double), ("norm_mode", c_int), ("norm_eps", c_float), ("sel_mode", c_int),
                 ("tau", c_float), ("keep_counts", c_void_p), ("keep_first", c_int), ("keep_last", c_int),
-                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p), ("fused_projections", c_int), ("rms_folded", c_int)]
+                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p), ("rms_folded", c_int)]
 
 
 class LayerWsLayout(Structure):
@@ -377,7 +377,7 @@ def dash_fold_norm_weight(W: torch.Tensor, rms_weight: torch.Tensor, out: Option
 
 
 def _projections_fit(shape) -> bool:
-    """True if this library's GEMMs take every projection of the block (256-column tiles, depth in steps of 64)."""
+    """True if every projection of the block runs with its fused epilogue (256-column tiles, depth in steps of 64)."""
     nq, hd = (shape.Hq + 2 * shape.Hkv) * shape.D, shape.Hq * shape.D
     ok = shape.d % 256 == 0 and nq % 256 == 0 and ((shape.Hq + shape.Hkv) * shape.D) % 256 == 0 and hd % 64 == 0
     return ok and (shape.m == 0 or shape.m % 128 == 0)
@@ -387,20 +387,21 @@ class Layer:
     """Device-resident weights and configuration of one block for dash_layer_step."""
 
     def __init__(self, shape, weights, device, norm_mode=NORM_REL, norm_eps=1e-12, sel_mode=SEL_THRESHOLD, tau=0.0,
-                 keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2, fused_projections=True):
+                 keep_counts: Optional[torch.Tensor] = None, keep_first=0, keep_last=0, scatter_which=2, fold_norms=True):
         self.shape = shape
         self.Wqkv = torch.cat([weights["Wq"], weights["Wk"], weights["Wv"]], dim=1).contiguous().to(device)
         self.Wo = weights["Wo"].contiguous().to(device)
         self.rms_w = weights["rms_w"].contiguous().to(device)
-        # with fused projections (bf16) the norm's weight is folded into the projection once, here, by the library: the step then
-        # needs no normalisation pass (the row factor 1 / rms is applied to the projection's accumulators)
-        self.rms_folded = bool(fused_projections) and self.Wqkv.dtype == torch.bfloat16 and _projections_fit(shape)
+        # where the projections run with their fused epilogues (bf16, whole 256-column tiles) the norm's weight is folded into the
+        # projection once, here, by the library: the step then needs no normalisation pass (the row factor 1 / rms is applied to the
+        # projection's accumulators).  fold_norms=False keeps the norm as a pass of its own.
+        self.rms_folded = bool(fold_norms) and self.Wqkv.dtype == torch.bfloat16 and _projections_fit(shape)
         if self.rms_folded:
             dash_fold_norm_weight(self.Wqkv, self.rms_w, out=self.Wqkv)
         self.keep_counts = keep_counts
         self.cfg = LayerCfg(shape.d, shape.Hq, shape.Hkv, shape.D, dtype_code(self.Wo), self.Wqkv.data_ptr(), self.Wo.data_ptr(),
                             self.rms_w.data_ptr(), shape.rms_eps, shape.rope_base, norm_mode, norm_eps, sel_mode, tau,
-                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None, int(bool(fused_projections)), int(self.rms_folded))
+                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None, int(self.rms_folded))
 
     def set_tau(self, tau: float):
         self.cfg.tau = float(tau)

@@ -50,16 +50,16 @@ def run_block(block, H, tok, pos, cu, max_seqlen, x_full, b):
 def _weights(sh, seed):
     W = dict(wl.layer_weights(sh, seed))
     W.update(wl.ffn_weights(sh, seed))
-    # norm weights that are not all ones: with fused projections the binding folds them into Wqkv and Wgu
+    # norm weights that are not all ones: folded into Wqkv and Wgu (dash_fold_norm_weight) or applied by the norms' own passes
     g = torch.Generator().manual_seed(seed + 1000)
     W["rms_w"] = (1.0 + 0.2 * torch.randn(sh.d, generator=g)).to(sh.dtype)
     W["rms2_w"] = (1.0 + 0.2 * torch.randn(sh.d, generator=g)).to(sh.dtype)
     return W
 
 
-@pytest.mark.parametrize("fused", [False, True], ids=["library_gemms", "fused_projections"])
+@pytest.mark.parametrize("fold", [False, True], ids=["norm_as_a_pass", "norm_folded"])
 @pytest.mark.parametrize("case", ["cfg1_fp32", "mini_bf16_varlen"])
-def test_block_step_matches_oracle_threshold(case, fused):
+def test_block_step_matches_oracle_threshold(case, fold):
     if case == "cfg1_fp32":
         w = wl.config1(T=512, seed=31)
     else:
@@ -74,7 +74,7 @@ def test_block_step_matches_oracle_threshold(case, fused):
     tau = oc.kth_largest(ref0["r"], K)
     ref = oc.block_step(H, W, w.cu, pos, sh, tau=tau)
 
-    block = dash.Block(sh, W, DEV, tau=tau, fused_projections=fused)
+    block = dash.Block(sh, W, DEV, tau=tau, fold_norms=fold)
     b = BlockBuffers(block, T, S)
     x_full = torch.full((T, sh.d), 9.0, dtype=sh.dtype, device=DEV)
     tok = torch.arange(T, dtype=torch.int32, device=DEV)
@@ -95,15 +95,15 @@ def test_block_step_matches_oracle_threshold(case, fused):
         assert_close_h1(b.H_next[:k].float().cpu().numpy(), ref["rows"][0], "H_next", bf)
 
 
-@pytest.mark.parametrize("fused", [False, True], ids=["library_gemms", "fused_projections"])
-def test_block_step_keep_count_rule_with_protected_tokens(fused):
+@pytest.mark.parametrize("fold", [False, True], ids=["norm_as_a_pass", "norm_folded"])
+def test_block_step_keep_count_rule_with_protected_tokens(fold):
     w = wl.config2(T=640, seed=33, shape=wl.MINI)
     sh, T = w.shape, w.T
     H, W = w.tensors["H"], _weights(sh, 33)
     pos = wl.positions(w.cu)
     K = oc.keep_count(T, 0.667, 64, 32, mode=1)                  # Appendix A: protected prefix / suffix
     kc = torch.tensor([K], dtype=torch.int32, device=DEV)
-    block = dash.Block(sh, W, DEV, sel_mode=dash.SEL_KEEP_COUNT, keep_counts=kc, keep_first=64, keep_last=32, fused_projections=fused)
+    block = dash.Block(sh, W, DEV, sel_mode=dash.SEL_KEEP_COUNT, keep_counts=kc, keep_first=64, keep_last=32, fold_norms=fold)
     b = BlockBuffers(block, T, 1)
     x_full = torch.zeros(T, sh.d, dtype=sh.dtype, device=DEV)
     run_block(block, H.to(DEV), torch.arange(T, dtype=torch.int32, device=DEV), pos.to(DEV), w.cu.to(DEV), T, x_full, b)
@@ -116,15 +116,15 @@ def test_block_step_keep_count_rule_with_protected_tokens(fused):
     assert torch.equal(b.H_next[:K].cpu(), x_full.cpu()[np.flatnonzero(mask)])
 
 
-@pytest.mark.parametrize("fused", [False, True], ids=["library_gemms", "fused_projections"])
-def test_block_step_qwen_shape_sampled_rows(fused):
+@pytest.mark.parametrize("fold", [False, True], ids=["norm_as_a_pass", "norm_folded"])
+def test_block_step_qwen_shape_sampled_rows(fold):
     w = wl.config2(T=2048, seed=34)
     sh, T = w.shape, w.T
     H, W = w.tensors["H"], _weights(sh, 34)
     pos = wl.positions(w.cu)
     rows = wl.sample_rows(w.cu, 40, seed=8).numpy()
     ref = oc.block_step(H, W, w.cu, pos, sh, attn_rows=rows)
-    block = dash.Block(sh, W, DEV, tau=0.0, fused_projections=fused)
+    block = dash.Block(sh, W, DEV, tau=0.0, fold_norms=fold)
     b = BlockBuffers(block, T, 1)
     x_full = torch.zeros(T, sh.d, dtype=sh.dtype, device=DEV)
     tok = torch.arange(T, dtype=torch.int32, device=DEV)
@@ -178,3 +178,37 @@ def test_block_step_block_signal_and_high_direction_ablations():
     assert int(b.n_next.item()) == K
     assert np.array_equal(m2, oc.select(r2, w.cu, oc.KEEP_COUNT, keep_counts=[K], halt_high=True))
     assert r2[m2 == 1].max() <= r2[m2 == 0].min()                           # the low scores stay, the high ones halt
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32], ids=["bf16", "fp32"])
+def test_block_step_shapes_without_whole_tiles(dtype):
+    """A block whose projections have no whole 256-column tiles and whose depth is no multiple of 64 (d = 520, 3 + 1 heads of 64,
+    FFN width 200): the same GEMM kernel runs them plain -- partial tiles zero-filled by the loads, columns past the edge not
+    stored -- with the norm, the rotary embedding, the residual and SwiGLU as passes of their own; fp32 tensors go through bf16
+    copies of the operands."""
+    sh = wl.LayerShape(d=520, Hq=3, Hkv=1, D=64, rope_base=1.0e4, dtype=dtype, m=200)
+    w = wl.config2(T=700, seed=37, shape=sh)
+    w.cu = wl.cu_from_lengths([257, 0, 443])
+    T, S = w.T, w.S
+    bf = dtype == torch.bfloat16
+    H, W = w.tensors["H"], _weights(sh, 37)
+    pos = wl.positions(w.cu)
+    ref0 = oc.block_step(H, W, w.cu, pos, sh, tau=0.0)
+    K = oc.keep_count(T, 0.4)
+    tau = oc.kth_largest(ref0["r"], K)
+    ref = oc.block_step(H, W, w.cu, pos, sh, tau=tau)
+    block = dash.Block(sh, W, DEV, tau=tau)
+    assert not block.layer.rms_folded and not block.rms2_folded
+    b = BlockBuffers(block, T, S)
+    x_full = torch.full((T, sh.d), 9.0, dtype=sh.dtype, device=DEV)
+    tok = torch.arange(T, dtype=torch.int32, device=DEV)
+    run_block(block, H.to(DEV), tok, pos.to(DEV), w.cu.to(DEV), 443, x_full, b)
+    r_gpu, mask = b.r.cpu().numpy(), b.mask.cpu().numpy()
+    assert np.max(np.abs(r_gpu - ref["r"]) / ref["r"]) < 2e-2
+    flips, _ = check_mask(mask, r_gpu, ref["r"], tau, w.cu)
+    assert_close_h1(x_full.float().cpu().numpy(), ref["H1"], "H' (x_full)", bf)
+    idx = np.flatnonzero(mask)
+    k = int(b.n_next.item())
+    assert k == idx.size and abs(k - K) <= flips
+    assert torch.equal(b.H_next[:k].cpu(), x_full.cpu()[idx])
+    assert np.array_equal(b.tok_next[:k].cpu().numpy(), idx)

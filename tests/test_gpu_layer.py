@@ -51,9 +51,9 @@ def check_mask(mask_gpu, r_gpu, r_ref, tau, cu, kf=0, kl=0):
     return int((mask_gpu != ref).sum()), int(band.sum())
 
 
-@pytest.mark.parametrize("fused", [False, True], ids=["library_gemms", "fused_projections"])
+@pytest.mark.parametrize("fold", [False, True], ids=["norm_as_a_pass", "norm_folded"])
 @pytest.mark.parametrize("cfg", ["cfg1", "mini_bf16", "mini_varlen"])
-def test_layer_step_matches_oracle(cfg, fused):
+def test_layer_step_matches_oracle(cfg, fold):
     if cfg == "cfg1":
         w = wl.config1()
     elif cfg == "mini_bf16":
@@ -64,7 +64,7 @@ def test_layer_step_matches_oracle(cfg, fused):
     sh = w.shape
     H, W = w.tensors["H"], dict(w.weights[0])
     if cfg != "cfg1":
-        # a norm weight that is not all ones: with fused projections the binding folds it into Wqkv
+        # a norm weight that is not all ones: folded into Wqkv by dash_fold_norm_weight, or applied by the norm's own pass
         W["rms_w"] = (1.0 + 0.2 * torch.randn(sh.d, generator=torch.Generator().manual_seed(9))).to(sh.dtype)
     T, S = w.T, w.S
     pos = wl.positions(w.cu)
@@ -73,7 +73,7 @@ def test_layer_step_matches_oracle(cfg, fused):
     tau = oc.kth_largest(ref0["r"], K)
     ref = oc.layer_step(H, W, w.cu, pos, sh, tau=tau)
 
-    layer = dash.Layer(sh, W, DEV, tau=tau, fused_projections=fused)
+    layer = dash.Layer(sh, W, DEV, tau=tau, fold_norms=fold)
     bufs = StepBuffers(layer, T, S, T, sh.dtype)
     x_full = torch.full((T, sh.d), 9.0, dtype=sh.dtype, device=DEV)
     tok = torch.arange(T, dtype=torch.int32, device=DEV)
@@ -88,9 +88,9 @@ def test_layer_step_matches_oracle(cfg, fused):
     assert_close_rms(QKV[:, (sh.Hq + sh.Hkv) * sh.D:], ref["V"].reshape(T, -1), "V", tol=4e-2)
     assert_close_rms(bufs.view(bufs.lay.O, T, sh.Hq * sh.D, sh.dtype).float().cpu().numpy(), ref["O"].reshape(T, -1), "attention O",
                      atol=(2.0 ** (math.floor(math.log2(float(np.abs(ref["V"]).max()))) - 8)) if sh.dtype == torch.bfloat16 else 0.0)
-    if sh.dtype == torch.float32 or not fused:
-        # with fused projections (bf16) the output projection adds the residual on its accumulators and U is never stored
-        # (r and H~ below are what it leaves)
+    if sh.dtype == torch.float32:
+        # with bf16 tensors and whole 256-column tiles the output projection adds the residual on its accumulators and U is never
+        # stored (r and H~ below are what it leaves)
         # U is an intermediate too (stored after O was stored): twice the bar, as for Q and K above
         assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype).float().cpu().numpy(), ref["U"], "U", tol=4e-2)
     # H~ of every entry token reaches x_full (threshold rule: score, residual, scatter and compaction run as one pass,
@@ -212,7 +212,7 @@ def test_layer_step_rows_beyond_the_packed_end_and_protected_tokens():
     Hp = torch.cat([H, torch.full((pad, sh.d), float("nan"), dtype=sh.dtype)])
     tokp = torch.cat([perm, torch.full((pad,), 0, dtype=torch.int32)])
     posp = torch.cat([pos, torch.zeros(pad, dtype=torch.int32)])
-    layer = dash.Layer(sh, W, DEV, tau=tau, keep_first=kf, keep_last=kl, fused_projections=True)
+    layer = dash.Layer(sh, W, DEV, tau=tau, keep_first=kf, keep_last=kl)
     bufs = StepBuffers(layer, T + pad, S, T + pad, sh.dtype)
     x_full = torch.full((T + pad, sh.d), 9.0, dtype=sh.dtype, device=DEV)
     run_step(layer, Hp.to(DEV), tokp.to(DEV), posp.to(DEV), w.cu.to(DEV), 443, x_full, bufs)
