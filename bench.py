@@ -210,6 +210,8 @@ def setup_block_step(args, dash, dev, rank):
     H_host, pos_host = _pin(w.tensors["H"]), _pin(wl.positions(w.cu))
     tok_host, cu_host = _pin(torch.arange(T, dtype=torch.int32)), _pin(w.cu)
     layer = dash.Layer(sh, w.weights[0], dev, tau=0.0)
+    if layer.rms_folded:       # the rotary angles by position: one table per prefill (shared by all its blocks), made outside the step
+        layer.set_handover(dash.dash_rope_table(sh.rope_base, sh.D, T, dev))
     B = StepBuffers(dash, layer, T, S, sh.d, sh.dtype, dev)
     H = torch.empty(T, sh.d, dtype=sh.dtype, device=dev)
     pos, tok = torch.empty(T, dtype=torch.int32, device=dev), torch.empty(T, dtype=torch.int32, device=dev)
@@ -300,8 +302,9 @@ def setup_block_step(args, dash, dev, rank):
     return {
         "workload": f"{name}, batch 1, seq {T}, threshold at the {int(w.rho * 100)}th percentile ({n_active} of {T} tokens stay active)",
         "dtype": "f32" if sh.dtype == torch.float32 else "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 6,
-        "launch_note": "per step: (a memset of the tail's look-back words,) attention item list, row factors + rotary angles, QKV GEMM (norm factor + "
-                       "rotary on the accumulators), attention, output GEMM (+ residual, score sums), tail (score + threshold + compaction)",
+        "launch_note": "per step: (a memset of the tail's look-back words,) attention item list, row factors of the norm (the rotary angles come "
+                       "from a table made once per prefill), QKV GEMM (norm factor + rotary on the accumulators), attention, output GEMM "
+                       "(+ residual, score sums), tail (score + threshold + compaction)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(*host_out),
         "extra": {"n_active_after": n_active, "tau": tau}, "e2e_pipeline": e2e_pipeline,
         "attn": (lambda: dash.dash_varlen_attention(Q, Kt, V, cu, T, O=Obuf, ws=attn_ws)), "attn_flops": attention_flops(w.cu.tolist(), sh.Hq, sh.D),
@@ -320,6 +323,11 @@ def setup_cascade(args, dash, dev, rank):
     sh, S, es = w.shape, w.S, 2
     Ks = [dash.dash_keep_count(T, 1.0 - f) for f in w.fractions]
     layers = [dash.Layer(sh, w.weights[l], dev, tau=0.0) for l in range(Lr)]
+    # handed from block to block: the rotary table of the prefill and the norm's row factors (layer l + 1 takes those layer l left)
+    table = dash.dash_rope_table(sh.rope_base, sh.D, T, dev)
+    inv = [torch.zeros(T, dtype=torch.float32, device=dev) for _ in range(2)]
+    for l in range(Lr):
+        layers[l].set_handover(table, inv[(l - 1) % 2] if l > 0 else None, inv[l % 2])
     A, Bb = StepBuffers(dash, layers[0], T, S, sh.d, sh.dtype, dev), StepBuffers(dash, layers[0], T, S, sh.d, sh.dtype, dev)
     H_host, pos_host = _pin(w.tensors["H"]), _pin(wl.positions(w.cu))
     tok_host, cu_host = _pin(torch.arange(T, dtype=torch.int32)), _pin(w.cu)
@@ -380,8 +388,9 @@ def setup_cascade(args, dash, dev, rank):
     fl_all = sum(attention_flops([0, n], sh.Hq, sh.D) for n in n_in)
     return {
         "workload": f"configs[2]: cascade of {Lr} Qwen2.5-7B-shaped layers, bf16, batch 1, seq {T}, tokens entering the layers {n_in}, "
-                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 6 * Lr,
-        "launch_note": f"{Lr} block steps of 6 kernels each",
+                    f"{got} active after the last", "dtype": "bf16", "step": step, "h2d": h2d, "d2h": d2h, "tokens": sum(n_in), "launches": 5 * Lr + 1,
+        "launch_note": f"{Lr} block steps of 5 kernels each (item list, QKV GEMM, attention, output GEMM, tail; the first also forms its row factors; "
+                       "rotary table made once per prefill, row factors handed from block to block)",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(x_full_h, tok_h, cu_h),
         "extra": {"tokens_entering_layers": n_in, "active_after_last": got, "attention_flops_per_step": fl_all,
                   "value_counts": "tokens entering each of the 8 layers, summed"},
@@ -485,6 +494,8 @@ def setup_stack(args, dash, dev, rank):
     K = dash.dash_keep_count(T, rho, 64, 32, 1)
     kc = torch.tensor([K], dtype=torch.int32, device=dev)
     blk = dash.Block(sh, Wt, dev, tau=0.0, keep_first=64, keep_last=32)   # one set of weights (timing only)
+    table = dash.dash_rope_table(sh.rope_base, sh.D, T, dev)              # once per prefill
+    inv = [torch.zeros(T, dtype=torch.float32, device=dev) for _ in range(2)]
     lay = dash.dash_block_workspace(blk, T, S)
     ws = dash.workspace(lay.total, dev)
     H_host, pos_host = _pin(wl.hidden_states(T, sh.d, rank_seed(5, rank), sh.dtype)), _pin(wl.positions(cu_h))
@@ -512,6 +523,7 @@ def setup_stack(args, dash, dev, rank):
             dst = bufs[(l - 1) % 2]
             select_here = halting and l == l_s
             blk.set_keep_counts(kc if select_here else None, dash.SEL_KEEP_COUNT if select_here else dash.SEL_THRESHOLD)
+            blk.set_handover(table, inv[l % 2] if l > 1 else None, inv[(l + 1) % 2])      # row factors handed from block to block
             dash.dash_block_step(blk, src["H"][:n_l], src["tok"][:n_l], src["pos"][:n_l], src["cu"], n_l, x_full, dst["H"], dst["tok"],
                                  dst["pos"], dst["cu"], n_next, r, mask, ws)
             src = dst
@@ -527,7 +539,7 @@ def setup_stack(args, dash, dev, rank):
     t_full = timer_simple(lambda: prefill(False), 2)
     t_dash = timer_simple(lambda: prefill(True), 2)
     # dominant kernel: the attention of a dense block (all T tokens); Q, K, V as the first block left them
-    h2d(); blk.set_keep_counts(None, dash.SEL_THRESHOLD)
+    h2d(); blk.set_keep_counts(None, dash.SEL_THRESHOLD); blk.set_handover(table)
     dash.dash_block_step(blk, H, tok, pos, cu, T, x_full, bufs[0]["H"], bufs[0]["tok"], bufs[0]["pos"], bufs[0]["cu"], n_next, r, mask, ws)
     torch.cuda.synchronize()
     nq = (sh.Hq + 2 * sh.Hkv) * sh.D
@@ -551,9 +563,10 @@ def setup_stack(args, dash, dev, rank):
     return {
         "workload": f"the paper's efficiency setting: {Lr} Qwen2.5-7B-shaped blocks with feed-forward, bf16, batch 1, seq {T}, single-shot selection "
                     f"at block {l_s}, compression ratio {rho}, first 64 / last 32 kept ({K} tokens stay); a step = the whole prefill",
-        "dtype": "bf16", "step": (lambda: prefill(True)), "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 9 * Lr + 1,
-        "launch_note": f"{Lr} block steps: (a memset,) attention item list, row factors + rotary angles, 4 GEMMs (rotary / residual + sums / SwiGLU / plain), "
-                       "attention, score from sums (+ select once), tail",
+        "dtype": "bf16", "step": (lambda: prefill(True)), "h2d": h2d, "d2h": d2h, "tokens": T, "launches": 8 * Lr + 2,
+        "launch_note": f"{Lr} block steps: (a memset,) attention item list, 4 GEMMs (rotary / residual + sums / SwiGLU / plain), attention, score from "
+                       "sums (+ select once), tail; the first block also forms its row factors; rotary table once per prefill, row factors "
+                       "handed from block to block",
         "h2d_bytes": _bytes(H_host, pos_host, tok_host, cu_host), "d2h_bytes": _bytes(x_h, tok_h), "extra": extra,
         "attn": (lambda: dash.dash_varlen_attention(Q, Kt, V, cu, T, O=Obuf, ws=attn_ws)), "attn_flops": attention_flops([0, T], sh.Hq, sh.D),
         "attn_name": f"attention_kernel<{sh.D}> (dense block, {T} tokens)",

@@ -255,6 +255,16 @@ typedef struct {
                                     * the norm costs no pass of its own -- one pass over H yields the row factors 1 / rms, which
                                     * the projection applies to its accumulators.  Only where the projections run with their
                                     * fused epilogues (see below); DASH_ERR_UNSUPPORTED otherwise. */
+    /* What a prefill can hand from block to block instead of recomputing it (all optional; they need rms_folded = 1,
+     * DASH_ERR_UNSUPPORTED otherwise):                                                                                   */
+    const void*  rope_table;       /* NULL, or the (cos, sin) pairs of dash_rope_table for positions 0 .. rope_table_len - 1 (same
+                                    * rope_base and D): the rotary angles of a row are looked up by its position instead of
+                                    * being formed in every block (positions beyond the table use its last entry) */
+    int64_t      rope_table_len;
+    const float* inv_rms_in;       /* NULL, or fp32 [n]: 1 / sqrt(mean(H_in[t]^2) + rms_eps) of every entering row, e.g. the
+                                    * inv_rms_next of the block step that produced H_in: no pass over H_in is needed then */
+    float*       inv_rms_next;     /* NULL, or fp32 [n]: receives that row factor for every row of H_next (from the sums the step
+                                    * has at hand), for the next block's inv_rms_in */
 } dash_layer_cfg;
 /* The projections (Wqkv, Wo; Wgu, Wd of dash_block_step) run in this library's tcgen05 GEMMs (256 x 256 tiles on CTA pairs).
  * bf16 tensors whose projections have whole 256-column tiles ((Hq + 2 Hkv) D, (Hq + Hkv) D and d multiples of 256, d and Hq D
@@ -273,6 +283,13 @@ typedef struct {
  * misaligned pointers, d < 1, N < 1, N not a multiple of 8 (bf16) / 4 (fp32), strides smaller than N. */
 int dash_fold_norm_weight(const void* W, const void* rms_weight, int d, int64_t N, int64_t ldw, dash_dtype dt,
                           void* W_out, int64_t ldo, void* stream);
+
+/* Rotary angles once per prefill (the rotary embedding inside Attn of Eq. 1; rotate-half pairs (i, i + D/2), angle
+ * pos * rope_base^(-2i/D)): table[pos * (D/2) + i] = (cos, sin) as two fp32, for pos = 0 .. n_pos - 1; the angle is formed and
+ * reduced in fp64, its sine and cosine evaluated in fp32.  table: device, n_pos * (D/2) * 8 bytes, 8-byte aligned.  A block
+ * step whose cfg.rope_table points here looks the angles up by position instead of forming them again in every block.
+ * Asynchronous on `stream`.  DASH_ERR_INVALID_ARG for a null table, n_pos < 1, rope_base <= 0 or D not in {64, 128}. */
+int dash_rope_table(double rope_base, int D, int64_t n_pos, void* table, void* stream);
 
 /* Byte offsets of the intermediates inside the workspace of dash_layer_step
  * (for inspection by tests and tools).  Ht (H~ = H + U) is only written when the

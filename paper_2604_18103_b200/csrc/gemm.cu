@@ -225,7 +225,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 // heads of D columns; inside a head of Q or K the pair (i, i + D/2) is rotated by the angle of (row, i)
                 __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.C) + (int64_t)row * g.ldc + nt * kGN;
                 const int D = g.e.D, half = D >> 1;
-                const float2* cs = g.e.rope_table + (int64_t)row * half;       // (cos, sin) of this row
+                int64_t trow = row;                                            // (cos, sin) of this row: its own entry, or its position's
+                if (g.e.rope_pos) { trow = live ? g.e.rope_pos[row] : 0; if (trow >= g.e.rope_len) trow = g.e.rope_len - 1; if (trow < 0) trow = 0; }
+                const float2* cs = g.e.rope_table + trow * half;
                 const float rsc = (g.e.row_scale && live) ? g.e.row_scale[row] : 1.0f;
                 for (int h0 = 0; h0 < kGN; h0 += D) {
                     const bool rotate = (nt * kGN + h0) < g.e.n_rot_cols;
@@ -351,14 +353,16 @@ row_prep_kernel(const int32_t* __restrict__ pos, int64_t n, int half, RopeFreqs 
                 }
             }
         }
-        const double ps = (double)pos[t];
-        for (int i = lane; i < half; i += 32) {
-            // angle formed and reduced to [-pi, pi] in fp64 (three operations), sine and cosine of the reduced angle in fp32
-            const double ang = ps * fr.inv_freq[i];
-            const double red = fma(-6.283185307179586476925286766559, rint(ang * 0.15915494309189533576888376337251), ang);
-            float sn, cs;
-            sincosf((float)red, &sn, &cs);
-            table[t * half + i] = make_float2(cs, sn);
+        if (table) {
+            const double ps = pos ? (double)pos[t] : (double)t;
+            for (int i = lane; i < half; i += 32) {
+                // angle formed and reduced to [-pi, pi] in fp64 (three operations), sine and cosine of the reduced angle in fp32
+                const double ang = ps * fr.inv_freq[i];
+                const double red = fma(-6.283185307179586476925286766559, rint(ang * 0.15915494309189533576888376337251), ang);
+                float sn, cs;
+                sincosf((float)red, &sn, &cs);
+                table[t * half + i] = make_float2(cs, sn);
+            }
         }
         if (inv_rms) {
             ss = warp_sum(ss);

@@ -14,6 +14,8 @@ struct GemmEpilogue {
     // rope_table [n, D/2] = (cos, sin) of every row
     int D = 0, n_rot_cols = 0;
     const float2* rope_table = nullptr;
+    // rope_pos null: the table holds one entry per row; else one per position and row t uses entry min(rope_pos[t], rope_len - 1)
+    const int32_t* rope_pos = nullptr; int64_t rope_len = 0;
     // ROPE, SWIGLU: row_scale (null: none) multiplies the accumulators of a row first -- 1 / rms(row) when the RMSNorm in front of the
     // projection is folded into it (its weight into W, its row factor here)
     const float* row_scale = nullptr;
@@ -37,7 +39,8 @@ int gemm_bf16(GemmEpilogueKind kind, const void* A, int64_t lda, const void* W, 
               int64_t K, const GemmEpilogue& e, const int32_t* n_dev, cudaStream_t st, bool out_f32 = false);
 // dst (bf16, row stride ld_dst) = src (fp32, row stride ld_src) rounded to nearest even; cols % 4 == 0
 int launch_f32_to_bf16(const float* src, int64_t ld_src, void* dst, int64_t ld_dst, int64_t rows, int64_t cols, cudaStream_t st);
-// per row: (cos, sin) of pos * base^(-2i/D) into table [n, D/2]; with inv_rms non-null also 1 / sqrt(mean(H_row^2) + eps) (bf16 H, row stride ldh)
+// per row: (cos, sin) of pos * base^(-2i/D) into table [n, D/2] (table null: not formed; pos null: the row number is the position);
+// with inv_rms non-null also 1 / sqrt(mean(H_row^2) + eps) (bf16 H, row stride ldh)
 int launch_row_prep(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const void* H, int64_t ldh, int d, float rms_eps,
                     float* inv_rms, const int32_t* n_dev, cudaStream_t st);
 

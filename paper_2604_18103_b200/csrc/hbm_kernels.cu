@@ -450,6 +450,7 @@ struct TailArgs {
     char* x_full; int64_t ldx_b; char* H_next; int64_t ldn_b;
     float* r_out; uint8_t* mask_out; int32_t* tok_next; int32_t* pos_next; int32_t* cu_next; int32_t* n_next;
     unsigned long long* tile_state; unsigned int* ticket; int* status;
+    float* inv_next; float inv_d, rms_eps;     // non-null: 1 / sqrt(mean(row^2) + rms_eps) of every row that goes to H_next, in its order
 };
 
 template <bool BF16>
@@ -458,6 +459,7 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
     constexpr int TILE = 32, NWARPS = kCompactThreads / 32, RPW = TILE / NWARPS;   // 2 rows per warp
     __shared__ int s_keep[TILE];
     __shared__ int s_src[TILE];
+    __shared__ float s_inv[TILE];
     __shared__ int s_base, s_count;
     __shared__ unsigned int s_tile, s_ballot;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -477,6 +479,7 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
         const int local = warp * RPW + rr;
         const int64_t row = t_start + local;
         int keep = 0;
+        float ss = 0.f;                                  // sum of squares of the row as it goes on (H~ or H')
         if (row < n) {
             float su = 0.f, sh = 0.f;
             if (a.U) {
@@ -496,7 +499,9 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
                         if (v < a.nvec) {
                             su += sumsq_vec<BF16>(x[k]);
                             sh += sumsq_vec<BF16>(y[k]);
-                            st_v4(o + ((int64_t)v << 4), add_vec<BF16>(x[k], y[k]));
+                            const uint4 z = add_vec<BF16>(x[k], y[k]);
+                            if (a.inv_next) ss += sumsq_vec<BF16>(z);
+                            st_v4(o + ((int64_t)v << 4), z);
                         }
                     }
                 }
@@ -507,7 +512,7 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
                 if (a.sums) {
                     // the projection's column tiles, summed in a fixed order (lane i takes tiles i, i + 32, ...)
                     su = 0.f; sh = 0.f;
-                    for (int i = lane; i < a.n_sum_tiles; i += 32) { const float4 p2 = a.sums[(int64_t)row * a.n_sum_tiles + i]; su += p2.x; sh += p2.y; }
+                    for (int i = lane; i < a.n_sum_tiles; i += 32) { const float4 p2 = a.sums[(int64_t)row * a.n_sum_tiles + i]; su += p2.x; sh += p2.y; ss += p2.z; }
                 }
                 su = warp_sum(su);
                 sh = warp_sum(sh);
@@ -520,7 +525,8 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
                 if (lane == 0) { a.r_out[row] = r; a.mask_out[row] = (uint8_t)keep; }
             }
         }
-        if (lane == 0) s_keep[local] = keep;
+        if (a.inv_next) ss = warp_sum(ss);
+        if (lane == 0) { s_keep[local] = keep; s_inv[local] = rsqrtf(ss * a.inv_d + a.rms_eps); }
     }
     __syncthreads();                                    // also orders this CTA's x_full rows before the copies below
     if (warp == 0) {
@@ -564,6 +570,7 @@ delta_tail_kernel(const TailArgs a, int64_t n_upper) {
             s_src[k] = t;
             a.tok_next[base + k] = a.tok_in[t];
             a.pos_next[base + k] = a.pos_in[t];
+            if (a.inv_next) a.inv_next[base + k] = s_inv[lane];
         }
         if (lane == 0) { s_base = base; s_count = agg; s_ballot = bal; }
     }
@@ -889,7 +896,8 @@ int clear_tail_ws(void* ws, size_t ws_bytes, int64_t n, cudaStream_t st) {
 int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float4* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
-                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, bool ws_is_clear, cudaStream_t st) {
+                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, bool ws_is_clear, cudaStream_t st, float* inv_next,
+                      float rms_eps) {
     const int es = dt == DASH_BF16 ? 2 : 4;
     if (!ws || ((uintptr_t)ws % 256) || ws_bytes < compact_ws_bytes(n)) return DASH_ERR_WORKSPACE;
     const int tiles = (int)((n + 31) / 32) > 0 ? (int)((n + 31) / 32) : 1;
@@ -901,6 +909,7 @@ int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, cons
     a.x_full = (char*)x_full; a.ldx_b = (int64_t)d * es; a.H_next = (char*)H_next; a.ldn_b = (int64_t)d * es;
     a.r_out = r_out; a.mask_out = mask_out; a.tok_next = tok_next; a.pos_next = pos_next; a.cu_next = cu_next; a.n_next = n_next;
     a.ticket = (unsigned int*)ws; a.tile_state = (unsigned long long*)((char*)ws + 256);
+    a.inv_next = inv_next; a.inv_d = 1.0f / (float)d; a.rms_eps = rms_eps;
     a.status = status_word_ptr();
     if (!a.status) return DASH_ERR_CUDA;
     if (dt == DASH_BF16) DASH_CUDA_TRY(launch_pdl(delta_tail_kernel<true>, tiles, kCompactThreads, 0, st, a, n));

@@ -116,7 +116,8 @@ int launch_sums_to_score(const float4* sums, int n_sum_tiles, int64_t n, dash_no
 int launch_delta_tail(const void* U, const void* H, const uint8_t* mask_in, const float4* sums, int n_sum_tiles, int64_t n, int d, dash_dtype dt, dash_norm_mode mode, float eps, float tau,
                       int keep_first, int keep_last, const int32_t* cu_in, int S, const int32_t* tok_in, const int32_t* pos_in,
                       void* x_full, void* H_next, float* r_out, uint8_t* mask_out, int32_t* tok_next, int32_t* pos_next,
-                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, bool ws_is_clear, cudaStream_t st);
+                      int32_t* cu_next, int32_t* n_next, void* ws, size_t ws_bytes, bool ws_is_clear, cudaStream_t st, float* inv_next,
+                      float rms_eps);
 int clear_tail_ws(void* ws, size_t ws_bytes, int64_t n, cudaStream_t st);
 int attention_plan(const int32_t* cu_seqlens, int S, int64_t n, int Hq, void* ws, size_t ws_bytes, cudaStream_t st);
 int attention_planned(const void* Q, const void* K, const void* V, void* O, float* lse, int64_t ldq, int64_t ldk, int64_t ldv, int64_t ldo,
@@ -215,6 +216,7 @@ static bool cfg_ok(const dash_layer_cfg* c) {
     if (c->scatter_which != 0 && c->scatter_which != 2) return false;
     if (!(c->rope_base > 0.0)) return false;
     if ((c->k_cache == nullptr) != (c->v_cache == nullptr)) return false;
+    if (c->rope_table && (c->rope_table_len < 1 || ((uintptr_t)c->rope_table % 8))) return false;
     return true;
 }
 
@@ -237,6 +239,11 @@ extern "C" int dash_fold_norm_weight(const void* W, const void* rms_weight, int 
     else fold_norm_weight_kernel<false><<<(int)blocks, 256, 0, st>>>((const char*)W, ldw * es, (const char*)rms_weight, (char*)W_out, ldo * es, d, (int)vpr);
     DASH_CUDA_TRY(cudaGetLastError());
     return DASH_OK;
+}
+
+extern "C" int dash_rope_table(double rope_base, int D, int64_t n_pos, void* table, void* stream) {
+    if (!table || ((uintptr_t)table % 8) || n_pos < 1 || n_pos > 0x7fffffffLL || !(rope_base > 0.0) || (D != 64 && D != 128)) return DASH_ERR_INVALID_ARG;
+    return launch_row_prep(nullptr, n_pos, D, rope_base, (float2*)table, nullptr, 0, 0, 0.f, nullptr, nullptr, (cudaStream_t)stream);
 }
 
 extern "C" int dash_layer_workspace(const dash_layer_cfg* cfg, int64_t n, int S, dash_layer_ws_layout* out) {
@@ -327,11 +334,19 @@ static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int
     GemmEpilogue e;
     e.D = D; e.n_rot_cols = (Hq + Hkv) * D; e.rope_table = W.rope_tab;
     const bool fused = bf && gemm_shape_ok(GEMM_ROPE, n, nq, d, d, nq, e);
+    if ((cfg->rope_table || cfg->inv_rms_in || cfg->inv_rms_next) && !(fused && cfg->rms_folded)) return DASH_ERR_UNSUPPORTED;
     if (fused && cfg->rms_folded) {
         // LN folded into the projection: its weight sits in Wqkv, its row factor 1 / rms is applied to the accumulators.
-        // One pass over H gives the row factors and the rotary angles; Q | K | V = (H Wqkv) / rms, Q and K rotated.
-        if ((rc = launch_row_prep(pos_in, n, D, cfg->rope_base, W.rope_tab, H_in, d, d, cfg->rms_eps, W.inv_rms, n_dev, st)) != DASH_OK) return rc;
-        e.row_scale = W.inv_rms;
+        // One pass over H gives the row factors and the rotary angles -- unless the caller hands them in (a table of the angles
+        // by position, made once per prefill; the row factors as the previous block left them): Q | K | V = (H Wqkv) / rms, Q and
+        // K rotated.
+        if (cfg->rope_table) { e.rope_table = (const float2*)cfg->rope_table; e.rope_pos = pos_in; e.rope_len = cfg->rope_table_len; }
+        if (!cfg->rope_table || !cfg->inv_rms_in) {
+            rc = launch_row_prep(pos_in, n, D, cfg->rope_base, cfg->rope_table ? nullptr : W.rope_tab, H_in, d, d, cfg->rms_eps,
+                                 cfg->inv_rms_in ? nullptr : W.inv_rms, n_dev, st);
+            if (rc != DASH_OK) return rc;
+        }
+        e.row_scale = cfg->inv_rms_in ? cfg->inv_rms_in : W.inv_rms;
         if ((rc = gemm_bf16(GEMM_ROPE, H_in, d, cfg->Wqkv, nq, W.QKV, nq, n, nq, d, e, n_dev, st)) != DASH_OK) return rc;
     } else if (fused) {
         // LN (read as RMSNorm), then Q | K | V = Hn Wqkv with the Q and K heads rotated on the accumulators
@@ -437,14 +452,16 @@ extern "C" int dash_layer_step(const dash_layer_cfg* cfg, const void* H_in, cons
             if (rc == DASH_OK)
                 return launch_delta_tail(nullptr, nullptr, nullptr, W.sums, d / 256, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau,
                                          cfg->keep_first, cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out,
-                                         tok_index_next, pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, true, st);
+                                         tok_index_next, pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, true, st,
+                                         cfg->inv_rms_next, cfg->rms_eps);
             if (rc != DASH_ERR_UNSUPPORTED) return rc;
             // fp32, or shapes without whole 256-column tiles: U through the plain GEMM, then r, H~, the rule, scatter and compaction in one pass
             if ((rc = out_proj_U(cfg, cu_in, S, n, W, st)) != DASH_OK) return rc;
             return launch_delta_tail(W.U, H_in, nullptr, nullptr, 0, n, d, cfg->dt, cfg->norm_mode, cfg->norm_eps, cfg->tau, cfg->keep_first,
                                      cfg->keep_last, cu_in, S, tok_index_in, pos_in, x_full, H_next, r_out, mask_out, tok_index_next,
-                                     pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, true, st);
+                                     pos_next, cu_next, n_next_dev, W.compact_ws, W.compact_bytes, true, st, nullptr, cfg->rms_eps);
         }
+        if (cfg->inv_rms_next) return DASH_ERR_UNSUPPORTED;      // the row factors come out of the fused tail pass (threshold rule, every row scattered)
         if ((rc = out_proj_U(cfg, cu_in, S, n, W, st)) != DASH_OK) return rc;
         if ((rc = score_and_select(cfg, H_in, cu_in, S, n, r_out, mask_out, W, st)) != DASH_OK) return rc;
         // updated states reach the full-length output (halted tokens stay frozen there from now on)
@@ -566,5 +583,5 @@ extern "C" int dash_block_step(const dash_block_cfg* cfg, const void* H_in, cons
     // for the tokens that stay, to the next block's packed buffer -- one pass, keep decisions taken from mask_out
     return launch_delta_tail(F, W.Ht, mask_out, nullptr, 0, n, d, a->dt, a->norm_mode, a->norm_eps, a->tau, a->keep_first, a->keep_last, cu_in, S,
                              tok_index_in, pos_in, x_full, H_next, nullptr, nullptr, tok_index_next, pos_next, cu_next, n_next_dev,
-                             W.compact_ws, W.compact_bytes, true, st);
+                             W.compact_ws, W.compact_bytes, true, st, a->inv_rms_next, a->rms_eps);
 }

@@ -31,7 +31,7 @@ EXPORTS = [
     "dash_delta_norm", "dash_select", "dash_compact", "dash_scatter", "dash_varlen_attention",
     "dash_layer_workspace", "dash_layer_step", "dash_workspace_bytes", "dash_compact_static",
     "dash_block_workspace", "dash_block_step", "dash_decode_attention", "dash_varlen_attention_indexed",
-    "dash_keep_counts_device", "dash_fold_norm_weight",
+    "dash_keep_counts_device", "dash_fold_norm_weight", "dash_rope_table",
 ]
 TEST_HOOKS = ["dash_testing_compact_stalled"]        # include/dash_testing.h
 COMPACT_STATIC_MAX_ROWS = 1 << 20
@@ -52,7 +52,8 @@ class LayerCfg(Structure):
                 ("Wqkv", c_void_p), ("Wo", c_void_p), ("rms_weight", c_void_p), ("rms_eps", c_float),
                 ("rope_base", c_double), ("norm_mode", c_int), ("norm_eps", c_float), ("sel_mode", c_int),
                 ("tau", c_float), ("keep_counts", c_void_p), ("keep_first", c_int), ("keep_last", c_int),
-                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p), ("rms_folded", c_int)]
+                ("scatter_which", c_int), ("k_cache", c_void_p), ("v_cache", c_void_p), ("rms_folded", c_int),
+                ("rope_table", c_void_p), ("rope_table_len", c_int64), ("inv_rms_in", c_void_p), ("inv_rms_next", c_void_p)]
 
 
 class LayerWsLayout(Structure):
@@ -106,6 +107,7 @@ def lib() -> ctypes.CDLL:
                                                                                   c_void_p, c_size_t, c_void_p]
         L.dash_keep_counts_device.argtypes = [c_void_p, c_int, c_double, c_int, c_int, c_int, c_void_p, c_void_p]
         L.dash_fold_norm_weight.argtypes = [c_void_p, c_void_p, c_int, c_int64, c_int64, c_int, c_void_p, c_int64, c_void_p]
+        L.dash_rope_table.argtypes = [c_double, c_int, c_int64, c_void_p, c_void_p]
         L.dash_layer_workspace.argtypes = [POINTER(LayerCfg), c_int64, c_int, POINTER(LayerWsLayout)]
         L.dash_layer_step.argtypes = [POINTER(LayerCfg), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_int64, c_int64,
                                       c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
@@ -376,6 +378,21 @@ def dash_fold_norm_weight(W: torch.Tensor, rms_weight: torch.Tensor, out: Option
     return out
 
 
+def dash_rope_table(rope_base: float, D: int, n_pos: int, device) -> torch.Tensor:
+    """(cos, sin) of pos * rope_base^(-2i/D) for pos < n_pos, i < D/2: fp32 [n_pos, D/2, 2], made once per prefill."""
+    table = torch.empty(n_pos, D // 2, 2, dtype=torch.float32, device=device)
+    _check(lib().dash_rope_table(float(rope_base), D, n_pos, _p(table), _stream()), "dash_rope_table")
+    return table
+
+
+def _set_handover(cfg, holder, rope_table, inv_rms_in, inv_rms_next):
+    holder._handover = (rope_table, inv_rms_in, inv_rms_next)           # keeps the tensors alive
+    cfg.rope_table = rope_table.data_ptr() if rope_table is not None else None
+    cfg.rope_table_len = rope_table.shape[0] if rope_table is not None else 0
+    cfg.inv_rms_in = inv_rms_in.data_ptr() if inv_rms_in is not None else None
+    cfg.inv_rms_next = inv_rms_next.data_ptr() if inv_rms_next is not None else None
+
+
 def _projections_fit(shape) -> bool:
     """True if every projection of the block runs with its fused epilogue (256-column tiles, depth in steps of 64)."""
     nq, hd = (shape.Hq + 2 * shape.Hkv) * shape.D, shape.Hq * shape.D
@@ -401,10 +418,16 @@ class Layer:
         self.keep_counts = keep_counts
         self.cfg = LayerCfg(shape.d, shape.Hq, shape.Hkv, shape.D, dtype_code(self.Wo), self.Wqkv.data_ptr(), self.Wo.data_ptr(),
                             self.rms_w.data_ptr(), shape.rms_eps, shape.rope_base, norm_mode, norm_eps, sel_mode, tau,
-                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None, int(self.rms_folded))
+                            keep_counts.data_ptr() if keep_counts is not None else None, keep_first, keep_last, scatter_which, None, None, int(self.rms_folded),
+                            None, 0, None, None)
 
     def set_tau(self, tau: float):
         self.cfg.tau = float(tau)
+
+    def set_handover(self, rope_table=None, inv_rms_in=None, inv_rms_next=None):
+        """What a prefill hands from block to block (needs the folded norm): the rotary table of dash_rope_table, the row factors
+        1 / rms of the entering rows (fp32 [n], a previous step's inv_rms_next) and a buffer for those of the rows that stay."""
+        _set_handover(self.cfg, self, rope_table, inv_rms_in, inv_rms_next)
 
     def set_kv_cache(self, k_cache: Optional[torch.Tensor], v_cache: Optional[torch.Tensor]):
         """[n, Hkv, D] buffers that receive this block's keys (rotary applied) and values, or None."""
@@ -445,6 +468,10 @@ class Block:
 
     def set_tau(self, tau: float):
         self.cfg.attn.tau = float(tau)
+
+    def set_handover(self, rope_table=None, inv_rms_in=None, inv_rms_next=None):
+        """As Layer.set_handover (the row factors handed on are those of H', the block's output)."""
+        _set_handover(self.cfg.attn, self, rope_table, inv_rms_in, inv_rms_next)
 
     def set_kv_cache(self, k_cache: Optional[torch.Tensor], v_cache: Optional[torch.Tensor]):
         """[n, Hkv, D] buffers that receive this block's keys (rotary applied) and values, or None."""

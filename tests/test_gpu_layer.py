@@ -137,8 +137,11 @@ def test_layer_step_keep_count_mode_and_protected_tokens():
     assert torch.equal(xf[mask == 0], Ht[mask == 0]) and (xf[mask == 1] == 9.0).all()
 
 
-def test_cascade_small_matches_oracle():
-    """Eight layers, per-layer keep fractions of the original T (multi-shot schedule), reduced T."""
+@pytest.mark.parametrize("handover", [False, True], ids=["recomputed", "handed_on"])
+def test_cascade_small_matches_oracle(handover):
+    """Eight layers, per-layer keep fractions of the original T (multi-shot schedule), reduced T.  handed_on: the rotary angles come
+    from one table made for the whole prefill and every block takes the norm's row factors from the block in front of it
+    (no pass over its input at all) instead of forming both itself."""
     T = 768
     w = wl.config3(T=T, seed=24, n_layers=8, shape=wl.MINI)
     sh = w.shape
@@ -163,8 +166,14 @@ def test_cascade_small_matches_oracle():
     x_full = torch.zeros(T, sh.d, dtype=sh.dtype, device=DEV)
     H, tok, pos, cu = w.tensors["H"].to(DEV), torch.arange(T, dtype=torch.int32, device=DEV), wl.positions(w.cu).to(DEV), w.cu.to(DEV)
     n_l, flipped = T, set()
+    if handover:
+        table = dash.dash_rope_table(sh.rope_base, sh.D, T, DEV)
+        inv = [torch.zeros(T, dtype=torch.float32, device=DEV) for _ in range(2)]
+        assert all(L.rms_folded for L in layers)
     for l in range(8):
         out = A if l % 2 == 0 else B
+        if handover:      # block 0 forms its own row factors; every later block gets them from the one in front
+            layers[l].set_handover(table, inv[(l - 1) % 2] if l > 0 else None, inv[l % 2])
         dash.dash_layer_step(layers[l], H[:n_l], tok[:n_l], pos[:n_l], cu, n_l, x_full, out.H_next, out.tok_next, out.pos_next,
                              out.cu_next, out.n_next, out.r, out.mask, out.ws)
         torch.cuda.synchronize()
@@ -193,6 +202,20 @@ def test_cascade_small_matches_oracle():
     got = x_full.float().cpu().numpy()[same]
     assert_close_rms(got, x_o[same], "x_full after the cascade", tol=2e-2 * math.sqrt(8))
     assert math.sqrt(float(np.mean((got - x_o[same]) ** 2))) < 1e-2
+
+
+def test_rope_table_holds_the_angles_of_every_position():
+    for base, D, n_pos in ((1.0e6, 128, 5000), (1.0e4, 64, 300)):
+        t = dash.dash_rope_table(base, D, n_pos, DEV).cpu().numpy().astype(np.float64)
+        ang = np.arange(n_pos, dtype=np.float64)[:, None] * base ** (-2.0 * np.arange(D // 2, dtype=np.float64) / D)[None, :]
+        assert np.max(np.abs(t[..., 0] - np.cos(ang))) < 1e-6 and np.max(np.abs(t[..., 1] - np.sin(ang))) < 1e-6
+    # the same rotation as the oracle's: a vector rotated with the table's entries
+    x = torch.randn(7, 1, 128, generator=torch.Generator().manual_seed(5), dtype=torch.float64).numpy()
+    pos = np.array([0, 1, 2, 100, 999, 4321, 4999])
+    t = dash.dash_rope_table(1.0e6, 128, 5000, DEV).cpu().numpy().astype(np.float64)[pos]
+    x1, x2 = x[:, 0, :64], x[:, 0, 64:]
+    mine = np.concatenate([x1 * t[..., 0] - x2 * t[..., 1], x2 * t[..., 0] + x1 * t[..., 1]], axis=-1)
+    assert np.max(np.abs(mine - oc.rope(x, pos, 1.0e6)[:, 0])) < 1e-5
 
 
 def test_layer_step_rows_beyond_the_packed_end_and_protected_tokens():
