@@ -9,7 +9,8 @@ from oracle import dash_oracle as oc
 from paper_2604_18103_b200 import dash
 from paper_2604_18103_b200 import workloads as wl
 from test_gpu_kernels import TOL, assert_close_rms
-from test_gpu_layer import BAND, check_mask
+from conftest import record_error
+from test_gpu_layer import BAND, _ratios, check_mask
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -82,6 +83,7 @@ def test_block_step_matches_oracle_threshold(case, fold):
     r_gpu, mask = b.r.cpu().numpy(), b.mask.cpu().numpy()
     assert np.max(np.abs(r_gpu - ref["r"]) / ref["r"]) < 2e-2
     flips, _ = check_mask(mask, r_gpu, ref["r"], tau, w.cu)
+    record_error(f"block step {case} {'folded' if fold else 'norm pass'} H'", *_ratios(x_full.float().cpu().numpy(), ref["H1"]))
     assert_close_h1(x_full.float().cpu().numpy(), ref["H1"], "H' (x_full)", bf)
     idx = np.flatnonzero(mask)
     k = int(b.n_next.item())
@@ -133,10 +135,12 @@ def test_block_step_qwen_shape_sampled_rows(fold):
     assert int(b.n_next.item()) == T
     r0 = b.r.cpu().numpy()
     assert np.max(np.abs(r0[rows] - ref["r"]) / ref["r"]) < 2e-2
-    # At this shape five bf16-stored stages lie between H~ and H' (norm output, gate | up, activation, F, H' itself; the oracle
-    # rounds nowhere): about 0.4 % of the row RMS per element, and the maximum over 39 x 3584 elements sits 4.6 sigma above
-    # that, at the 2e-2 bar itself (one element in 140 000 passed it by 1.8e-3).  Computation term for this test: 3e-2 x RMS.
-    assert_close_h1(x_full[rows].float().cpu().numpy(), ref["H1"], "H' (sampled rows)", tol=3e-2)
+    # H' at the bar of every H' check: 2e-2 x RMS for the computation plus the half-ulps of the two stores of the residual stream
+    # (measured here: 0.023 - 0.026 x RMS before, 0.015 - 0.017 x RMS after taking those half-ulps off)
+    record_error(f"block step Qwen shape H' (sampled rows, {'folded' if fold else 'norm pass'})", *_ratios(x_full[rows].float().cpu().numpy(), ref["H1"]))
+    record_error(f"block step Qwen shape H' minus the two stores' half-ulps ({'folded' if fold else 'norm pass'})",
+                 *_ratios(np.sign(x_full[rows].float().cpu().numpy() - ref["H1"]) * np.maximum(np.abs(x_full[rows].float().cpu().numpy() - ref["H1"]) - 2.0 ** -7 * np.abs(ref["H1"]), 0.0) + ref["H1"], ref["H1"]))
+    assert_close_h1(x_full[rows].float().cpu().numpy(), ref["H1"], "H' (sampled rows)")
     K = oc.keep_count(T, 0.4)
     tau = float(np.sort(r0)[::-1][K - 1])
     block.set_tau(tau)

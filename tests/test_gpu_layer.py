@@ -9,6 +9,7 @@ import torch
 from oracle import dash_oracle as oc
 from paper_2604_18103_b200 import dash
 from paper_2604_18103_b200 import workloads as wl
+from conftest import record_error
 from test_gpu_kernels import assert_close_rms
 
 pytestmark = pytest.mark.gpu
@@ -39,6 +40,14 @@ def run_step(layer, H, tok, pos, cu, max_seqlen, x_full, bufs):
                          bufs.cu_next, bufs.n_next, bufs.r, bufs.mask, bufs.ws)
     torch.cuda.synchronize()
     assert dash.dash_check_status() == dash.OK
+
+
+def _ratios(got, ref):
+    """(max |err| / RMS of the whole reference tensor, worst row's max |err| / RMS of that row)."""
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    g2, r2 = got.reshape(-1, got.shape[-1]), ref.reshape(-1, ref.shape[-1])
+    err = np.max(np.abs(g2 - r2), axis=1)
+    return float(err.max() / math.sqrt(float(np.mean(r2 * r2)))), float(np.max(err / np.maximum(np.sqrt(np.mean(r2 * r2, axis=1)), 1e-30)))
 
 
 def check_mask(mask_gpu, r_gpu, r_ref, tau, cu, kf=0, kl=0):
@@ -81,18 +90,23 @@ def test_layer_step_matches_oracle(cfg, fold):
 
     nq = (sh.Hq + 2 * sh.Hkv) * sh.D
     QKV = bufs.view(bufs.lay.QKV, T, nq, sh.dtype).float().cpu().numpy()
-    # intermediates (not outputs of the step): Q and K are rounded to the storage type twice
-    # (projection, then rotation), so they get twice the bar of the outputs
-    assert_close_rms(QKV[:, :sh.Hq * sh.D], ref["Q"].reshape(T, -1), "Q (rotary applied)", tol=4e-2)
-    assert_close_rms(QKV[:, sh.Hq * sh.D:(sh.Hq + sh.Hkv) * sh.D], ref["K"].reshape(T, -1), "K (rotary applied)", tol=4e-2)
-    assert_close_rms(QKV[:, (sh.Hq + sh.Hkv) * sh.D:], ref["V"].reshape(T, -1), "V", tol=4e-2)
+    tag = f"layer step {cfg} {'folded' if fold else 'norm pass'}"
+    record_error(f"{tag} Q", *_ratios(QKV[:, :sh.Hq * sh.D], ref["Q"].reshape(T, -1)))
+    record_error(f"{tag} K", *_ratios(QKV[:, sh.Hq * sh.D:(sh.Hq + sh.Hkv) * sh.D], ref["K"].reshape(T, -1)))
+    record_error(f"{tag} V", *_ratios(QKV[:, (sh.Hq + sh.Hkv) * sh.D:], ref["V"].reshape(T, -1)))
+    record_error(f"{tag} O", *_ratios(bufs.view(bufs.lay.O, T, sh.Hq * sh.D, sh.dtype).float().cpu().numpy().reshape(T, sh.Hq, sh.D), ref["O"]))
+    record_error(f"{tag} H~", *_ratios(x_full.float().cpu().numpy(), ref["Ht"]))
+    # intermediates of the step, held to the bar of its outputs: Q and K come out of the projection's accumulators rotated and are
+    # rounded to the storage type once (measured: at most 0.018 x RMS, V included)
+    assert_close_rms(QKV[:, :sh.Hq * sh.D], ref["Q"].reshape(T, -1), "Q (rotary applied)")
+    assert_close_rms(QKV[:, sh.Hq * sh.D:(sh.Hq + sh.Hkv) * sh.D], ref["K"].reshape(T, -1), "K (rotary applied)")
+    assert_close_rms(QKV[:, (sh.Hq + sh.Hkv) * sh.D:], ref["V"].reshape(T, -1), "V")
     assert_close_rms(bufs.view(bufs.lay.O, T, sh.Hq * sh.D, sh.dtype).float().cpu().numpy(), ref["O"].reshape(T, -1), "attention O",
                      atol=(2.0 ** (math.floor(math.log2(float(np.abs(ref["V"]).max()))) - 8)) if sh.dtype == torch.bfloat16 else 0.0)
     if sh.dtype == torch.float32:
         # with bf16 tensors and whole 256-column tiles the output projection adds the residual on its accumulators and U is never
         # stored (r and H~ below are what it leaves)
-        # U is an intermediate too (stored after O was stored): twice the bar, as for Q and K above
-        assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype).float().cpu().numpy(), ref["U"], "U", tol=4e-2)
+        assert_close_rms(bufs.view(bufs.lay.U, T, sh.d, sh.dtype).float().cpu().numpy(), ref["U"], "U")
     # H~ of every entry token reaches x_full (threshold rule: score, residual, scatter and compaction run as one pass,
     # which writes H~ there and nowhere else); tok is the identity here
     assert_close_rms(x_full.float().cpu().numpy(), ref["Ht"], "H~ (x_full)")
