@@ -3,10 +3,12 @@
 // HBM-bound: every cached key/value row is read once.  The G = Hq / Hkv query heads that share one KV
 // head form the (mostly empty) 128-row operand of the tcgen05 MMAs, so K and V tiles stream through
 // shared memory once per KV head; the keys of a sequence are split over persistent CTAs (flash-decoding),
-// whose partial (max, sum, O) results a small merge kernel combines.
-//   plan kernel   : items (sequence, KV head, key-block range), sized so that one item exists per CTA (batches of up to 32 sequences: the CTAs plan for themselves) or four per SM (handed out by ticket)
-//   decode kernel : per item  S = Q K_j^T -> masked online softmax (one warp: the rows that exist) -> O += P V_j
-//   merge kernel  : O = sum_i 2^((m_i - m) c) O_i / sum_i 2^((m_i - m) c) l_i
+// one per SM, and the CTA that finishes the last split of a (sequence, KV head) combines the partial (max, sum, O) results:
+// one kernel per call (behind a memset of the per-head arrival counters) for batches of up to 32 sequences.
+//   items         : (sequence, KV head, key-block range), sized so that one item exists per CTA where that keeps the CTAs busy
+//                   (up to 32 sequences: the CTAs plan for themselves; larger batches: a one-CTA plan kernel in front)
+//   per item      : S = Q K_j^T -> masked online softmax (one warp: the rows that exist) -> O += P V_j
+//   merge         : O = sum_i 2^((m_i - m) c) O_i / sum_i 2^((m_i - m) c) l_i
 #include <math.h>
 
 #include "common.cuh"
@@ -17,10 +19,12 @@ namespace dash {
 using namespace ptx;
 
 constexpr int kDecBN = 128;                  // keys per block
-constexpr int kDecThreads = 64;              // warp 0: softmax (rows 0..31 of the tile, G of them real), warp 1: TMA + MMA issue
+constexpr int kDecThreads = 256;             // warp 0: softmax (rows 0..31 of the tile, G of them real), warp 1: TMA + MMA issue, all eight: merge
 constexpr int kDecRows = 8;                  // query heads per KV head the tile can hold (box of the Q load)
+constexpr int kDecRing = 5;                  // K / V tile buffers
 constexpr long long kDecWaitCycles = 4000000000LL;
-constexpr uint32_t kDecTmemCols = 256;       // S | O
+constexpr uint32_t kDecTmemCols = 512;       // S_0 | S_1 | O (| unused)
+constexpr int kMergeMaxSplits = 640;         // key splits of one (sequence, KV head) the merge can weigh; the plans stay below
 
 struct DecItem { int s, kvh, b0, b1; };
 
@@ -28,21 +32,22 @@ struct DecParams {
     const int32_t* cu;
     int S, Hq, Hkv, G;
     float scale_log2, scale;
-    float* partial;             // [item][kDecRows][D + 2]: unnormalised O row, then m, l
+    float* partial;             // [item][kDecRows][D + 4]: unnormalised O row, then m, l
     const DecItem* plan;        // null: the CTAs plan for themselves (S <= kSelfPlanSeqs)
+    const int2* seg;            // with a plan: first item and number of items of every (sequence, KV head)
     const int* n_items;
-    unsigned int* ticket;
+    unsigned int* counters;     // [S][Hkv] items finished, zero at launch
     int target;                 // items aimed at (self-planning)
     int* status;
+    void* out; int64_t ldo; float* lse;
 };
 
-// Batches of up to kSelfPlanSeqs sequences need no plan kernel, no ticket and no scratch clear: every CTA derives the chunk
-// length and its items (item i -> CTA i mod grid; the items are equally long) from cu_seqlens itself, and so does the merge.
+// Batches of up to kSelfPlanSeqs sequences need no plan kernel: every CTA derives the chunk length and its items
+// (item i -> CTA i mod grid; the items are equally long) from cu_seqlens itself.
 constexpr int kSelfPlanSeqs = 32;
 __device__ __forceinline__ int dec_blocks(const int32_t* cu, int s) { return (cu[s + 1] - cu[s] + kDecBN - 1) / kDecBN; }
 // The plan of a self-planning launch, built once per CTA in shared memory: thread s fetches sequence s, thread 0 does the few
-// serial steps over at most kSelfPlanSeqs numbers.  (Every thread deriving it on its own from cu_seqlens cost the merge kernel of a
-// 32-sequence batch more than its merging.)
+// serial steps over at most kSelfPlanSeqs numbers.
 struct SelfPlan {
     int nb[kSelfPlanSeqs];        // key blocks of sequence s
     int first[kSelfPlanSeqs];     // first item of sequence s (its Hkv heads follow each other, `per` items each)
@@ -103,7 +108,7 @@ __device__ __forceinline__ DecItem self_plan_item(const SelfPlan& sp, int S, int
 // `target` items exist, then the items of every (sequence, KV head) written next to each other.
 __global__ void __launch_bounds__(256)
 decode_plan_kernel(const int32_t* __restrict__ cu, int S, int Hkv, int target, DecItem* __restrict__ plan, int2* __restrict__ seg,
-                   int* __restrict__ n_items, unsigned int* __restrict__ ticket, int max_items, int* __restrict__ seq_first) {
+                   int* __restrict__ n_items, unsigned int* __restrict__ counters, int max_items, int* __restrict__ seq_first) {
     __shared__ unsigned long long s_total;
     __shared__ int s_chunk;
     if (threadIdx.x == 0) s_total = 0;
@@ -124,7 +129,6 @@ decode_plan_kernel(const int32_t* __restrict__ cu, int S, int Hkv, int target, D
             k += ((nb + s_chunk - 1) / s_chunk) * Hkv;
         }
         *n_items = k < max_items ? k : max_items;
-        *ticket = 0u;
     }
     __syncthreads();
     const int chunk = s_chunk;
@@ -139,18 +143,78 @@ decode_plan_kernel(const int32_t* __restrict__ cu, int S, int Hkv, int target, D
             plan[first + i] = it;
         }
         seg[sh] = make_int2(first, cnt);
+        counters[sh] = 0u;
     }
 }
 
 template <int D>
 struct DecSmem {
     static constexpr int kTileBytes = kDecBN * D * 2;
-    static constexpr int kQ = 0, kK = kTileBytes, kV = 2 * kTileBytes, kBars = 3 * kTileBytes;
-    static constexpr int kTotal = kBars + 128;
+    static constexpr int kQ = 0, kRing = kTileBytes, kBars = (1 + kDecRing) * kTileBytes;
+    static constexpr int kTotal = kBars + 256;
 };
 
+// O and lse of a sequence without cached keys: zeros and -inf (what the sum over no keys is)
+template <bool OUT_F32>
+__device__ __forceinline__ void decode_write_empty(int s, int Hq, int D, void* out, int64_t ldo, float* lse) {
+    for (int i = threadIdx.x; i < Hq * D; i += blockDim.x) {
+        if (OUT_F32) reinterpret_cast<float*>(out)[(int64_t)s * ldo + i] = 0.f;
+        else reinterpret_cast<__nv_bfloat16*>(out)[(int64_t)s * ldo + i] = __float2bfloat16(0.f);
+    }
+    if (lse) for (int h = threadIdx.x; h < Hq; h += blockDim.x) lse[(int64_t)s * Hq + h] = -INFINITY;
+}
+__global__ void __launch_bounds__(128)
+decode_empty_kernel(int Hq, int D, void* out, int64_t ldo, float* lse) { decode_write_empty<false>((int)blockIdx.x, Hq, D, out, ldo, lse); }
+
+// The last CTA to finish an item of (sequence, KV head) combines that head group's partial results (G rows, `cnt` key splits starting
+// at item `first`): warp w takes row w -- the common maximum and the splits' weights over its lanes, then lane c the columns 4c..4c+3.
 template <int D>
-__global__ void __launch_bounds__(kDecThreads)
+__device__ __forceinline__ void decode_merge(const DecParams& p, float (*s_w)[kMergeMaxSplits], int s, int kvh, int first, int cnt) {
+    const int lane = threadIdx.x & 31, row = threadIdx.x >> 5;
+    if (row >= p.G) return;
+    constexpr int kRow = D + 4;
+    const size_t stride = (size_t)kDecRows * kRow;
+    const float* base = p.partial + ((size_t)first * kDecRows + row) * kRow;
+    float mx = -INFINITY;
+    for (int i = lane; i < cnt; i += 32) mx = fmaxf(mx, __ldcg(base + i * stride + D));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float ls = 0.f;
+    for (int i = lane; i < cnt; i += 32) {
+        const float wi = exp2f((__ldcg(base + i * stride + D) - mx) * p.scale_log2);
+        s_w[row][i] = wi;
+        ls += wi * __ldcg(base + i * stride + D + 1);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+    __syncwarp();
+    const int h = kvh * p.G + row;
+    if (4 * lane < D) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* col = base + 4 * lane;
+#pragma unroll 16
+        for (int i = 0; i < cnt; ++i) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(col + i * stride));
+            const float wi = s_w[row][i];
+            acc.x = fmaf(wi, v.x, acc.x); acc.y = fmaf(wi, v.y, acc.y); acc.z = fmaf(wi, v.z, acc.z); acc.w = fmaf(wi, v.w, acc.w);
+        }
+        const float inv = 1.0f / ls;
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)s * p.ldo + (int64_t)h * D + 4 * lane;
+        uint2 packed;
+        packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+        packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(o) = packed;
+    }
+    if (p.lse && lane == 0) p.lse[(int64_t)s * p.Hq + h] = mx * p.scale + logf(ls);
+}
+
+// One CTA per SM.  Warp 1 (one lane) streams the K and V tiles of the CTA's items, in order K_0 V_0 K_1 V_1 .. across the items,
+// through a ring of kDecRing tile buffers -- the loads run up to kDecRing tiles ahead of the MMAs, whatever item they belong to --
+// and issues the MMAs: S_g = Q K_g^T into one of two TMEM buffers (so S_{g+1} runs while warp 0 forms P_g), then O += P_g V_g.
+// Warp 0 is the softmax warp.  At the end of an item all eight warps meet: the CTA that completes the last item of a
+// (sequence, KV head) merges its splits and writes the output rows.
+template <int D>
+__global__ void __launch_bounds__(kDecThreads, 1)
 decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
               const __grid_constant__ CUtensorMap mapV, const DecParams p, int q_box_heads) {
     extern __shared__ uint8_t smem_raw[];
@@ -158,24 +222,31 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     constexpr int KCH = D / 64;
     constexpr int kChunkBytes = kDecBN * 128;
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = smem_base + L::kQ, sK = smem_base + L::kK, sV = smem_base + L::kV;
+    const uint32_t sQ = smem_base + L::kQ, sRing = smem_base + L::kRing;
     const uint32_t bars = smem_base + L::kBars;
-    const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_o = bars + 32, bar_p0 = bars + 40, bar_p1 = bars + 48;
-    const uint32_t tmem_slot = bars + 64;
+    const uint32_t bar_q = bars, bar_full = bars + 8 /* kDecRing of them */, bar_s = bars + 64 /* 2 */, bar_o = bars + 80 /* 2 */,
+                   bar_p0 = bars + 96 /* 2 */, bar_p1 = bars + 112 /* 2 */;
+    const uint32_t tmem_slot = bars + 128;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 64);
-    volatile uint32_t* abort_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 68);
-    volatile int* item_gen = reinterpret_cast<volatile int*>(smem_gen + L::kBars + 72);
+    volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 128);
+    volatile uint32_t* abort_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 132);
+    volatile int* last_gen = reinterpret_cast<volatile int*>(smem_gen + L::kBars + 136);
+    __shared__ SelfPlan sp;
+    __shared__ float s_w[kDecRows][kMergeMaxSplits];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    pdl_launch_dependents();                 // the merge kernel may get onto the SMs while this one runs
+    pdl_launch_dependents();
 
     // rows of the Q tile that no load ever writes must not hold NaN patterns: clear the tile once
     for (int i = tid * 16; i < L::kTileBytes; i += kDecThreads * 16) *reinterpret_cast<uint4*>(smem_gen + L::kQ + i) = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
     if (warp == 1) {
         if (lane == 0) {
-            mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1);
-            mbar_init(bar_s, 1); mbar_init(bar_o, 1); mbar_init(bar_p0, 32); mbar_init(bar_p1, 32);
+            mbar_init(bar_q, 1);
+            for (int i = 0; i < kDecRing; ++i) mbar_init(bar_full + 8 * i, 1);
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(bar_s + 8 * i, 1); mbar_init(bar_o + 8 * i, 1);
+                mbar_init(bar_p0 + 8 * i, 32); mbar_init(bar_p1 + 8 * i, 32);
+            }
             *abort_gen = 0;
             fence_barrier_init();
             fence_proxy_async_smem();
@@ -188,99 +259,151 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    pdl_wait();                              // set-up done; from here on the kernel in front has completed
+    pdl_wait();                              // set-up done; from here on the work in front on the stream has completed
     const uint32_t tmem = *tmem_slot_gen;
-    const uint32_t tS = tmem, tP = tmem, tO = tmem + 128;
+    const uint32_t tO = tmem + 256;          // S_0 / P_0 at column 0, S_1 / P_1 at 128, O at 256
     constexpr uint32_t idesc_s = idesc_bf16_f32(128, kDecBN, false, false);
     constexpr uint32_t idesc_o = idesc_bf16_f32(128, D, false, true);
     const bool self_plan = (p.plan == nullptr);
-    __shared__ SelfPlan sp;
     if (self_plan) self_plan_build(sp, p.cu, p.S, p.Hkv, p.target);
     const int n_items = self_plan ? sp.n_items : *p.n_items;
-    uint32_t blk0 = 0, items_done = 0;       // barrier phases run on across the items of this CTA
+    auto get_item = [&](int item) -> DecItem { return self_plan ? self_plan_item(sp, p.S, p.Hkv, item) : p.plan[item]; };
+    // sequences without cached keys have no item: their rows are written here
+    for (int s = (int)blockIdx.x; s < p.S; s += (int)gridDim.x)
+        if (p.cu[s + 1] - p.cu[s] <= 0) decode_write_empty<false>(s, p.Hq, D, p.out, p.ldo, p.lse);
 
-    for (;;) {
-        int item;
-        if (self_plan) {
-            item = (int)blockIdx.x + (int)items_done * (int)gridDim.x;
-        } else {
-            if (tid == 0) *item_gen = (int)atomicAdd(p.ticket, 1u);
-            __syncthreads();
-            item = *item_gen;
+    // ---- state of the issuing lane (warp 1, lane 0); g counts the key blocks of this CTA across its items ----
+    uint32_t loaded = 0;                     // tiles whose load has been issued (tile 2g: K of block g, 2g + 1: V)
+    uint32_t s_issued = 0, pv_issued = 0;    // blocks whose S / PV MMAs have been issued
+    uint32_t s_conf = 0, o_conf = 0;         // blocks whose S / PV MMAs are known to be complete (barrier phases taken in order)
+    int ld_round = 0, ld_j = 0, ld_nblk = 0, ld_row0 = 0, ld_kvh = 0;   // load cursor: item blockIdx.x + ld_round * gridDim.x, block ld_j of it
+    bool ld_more = false, prod_ok = true;
+    const bool producer = (warp == 1 && lane == 0);
+    auto ld_open = [&]() {                   // point the cursor at the first block of item ld_round (if there is one)
+        const int item = (int)blockIdx.x + ld_round * (int)gridDim.x;
+        ld_more = item < n_items;
+        if (ld_more) {
+            const DecItem it = get_item(item);
+            ld_j = 0; ld_nblk = it.b1 - it.b0; ld_kvh = it.kvh;
+            ld_row0 = p.cu[it.s] + it.b0 * kDecBN;
         }
-        if (item >= n_items || *abort_gen) break;
+    };
+    // block h's S MMAs are complete (each phase of bar_s[h & 1] is taken exactly once, in order: S_{h+2} is not issued before)
+    auto confirm_s = [&](uint32_t h) -> bool {
+        while (s_conf <= h) {
+            if (!mbar_wait(bar_s + 8 * (s_conf & 1), (s_conf >> 1) & 1, kDecWaitCycles)) return false;
+            ++s_conf;
+        }
+        return true;
+    };
+    auto confirm_o = [&](uint32_t h) -> bool {
+        while (o_conf <= h) {
+            if (!mbar_wait(bar_o + 8 * (o_conf & 1), (o_conf >> 1) & 1, kDecWaitCycles)) return false;
+            ++o_conf;
+        }
+        return true;
+    };
+    // issue loads while a ring buffer is free: tile t takes the buffer of tile t - kDecRing, free once the MMAs that read it are done
+    auto pump = [&]() -> bool {
+        while (ld_more) {
+            const uint32_t t = loaded;
+            if (t >= (uint32_t)kDecRing) {
+                const uint32_t prev = t - kDecRing, gp = prev >> 1;
+                if (prev & 1) { if (gp >= pv_issued) return true; if (!confirm_o(gp)) return false; }
+                else          { if (gp >= s_issued) return true;  if (!confirm_s(gp)) return false; }
+            }
+            const uint32_t slot = t % kDecRing, dst = sRing + slot * L::kTileBytes, bar = bar_full + 8 * slot;
+            mbar_arrive_expect_tx(bar, L::kTileBytes);
+            const CUtensorMap* map = (t & 1) ? &mapV : &mapK;
+            for (int c = 0; c < KCH; ++c) tma_load_3d(dst + c * kChunkBytes, map, bar, c * 64, ld_kvh, ld_row0 + ld_j * kDecBN);
+            ++loaded;
+            if (t & 1) {                     // V of the block: on to the next block, or the next item
+                if (++ld_j == ld_nblk) { ++ld_round; ld_open(); }
+            }
+        }
+        return true;
+    };
+    auto wait_full = [&](uint32_t t) -> bool { return mbar_wait(bar_full + 8 * (t % kDecRing), (t / kDecRing) & 1, kDecWaitCycles); };
+    auto issue_q = [&](const DecItem& it) {
+        mbar_arrive_expect_tx(bar_q, (uint32_t)(KCH * q_box_heads * 128));
+        for (int c = 0; c < KCH; ++c) tma_load_3d(sQ + c * kChunkBytes, &mapQ, bar_q, c * 64, it.kvh * p.G, it.s);
+    };
+    // O += P_h V_h (first of the item: O = ..); the first 64 keys of P start while the rest is still being formed
+    auto issue_pv = [&](uint32_t h, bool accumulate) -> bool {
+        const uint32_t b = h & 1, php = (h >> 1) & 1, tP = tmem + b * 128;
+        if (h >= 2 && !confirm_o(h - 2)) return false;                     // keeps the phases of bar_o[b] from running ahead of this lane
+        if (!mbar_wait(bar_p0 + 8 * b, php, kDecWaitCycles) || !wait_full(2 * h + 1)) return false;
+        const uint32_t sV = sRing + ((2 * h + 1) % kDecRing) * L::kTileBytes;
         tc_fence_after();
-        const DecItem it = self_plan ? self_plan_item(sp, p.S, p.Hkv, item) : p.plan[item];
+#pragma unroll
+        for (int kk = 0; kk < kDecBN / 32; ++kk)
+            mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, accumulate || (kk > 0));
+        if (!mbar_wait(bar_p1 + 8 * b, php, kDecWaitCycles)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = kDecBN / 32; kk < kDecBN / 16; ++kk)
+            mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, 1);
+        tc_commit(bar_o + 8 * b);
+        pv_issued = h + 1;
+        return true;
+    };
+    if (producer) {
+        ld_open();
+        if (ld_more) issue_q(get_item((int)blockIdx.x));
+        prod_ok = pump();
+    }
+
+    uint32_t g0 = 0, items_done = 0;         // first key block of the current item in the CTA's count; items finished
+    for (;;) {
+        const int item = (int)blockIdx.x + (int)items_done * (int)gridDim.x;
+        if (item >= n_items || *abort_gen) break;
+        const DecItem it = get_item(item);
         const int seq_a = p.cu[it.s], len = p.cu[it.s + 1] - seq_a;
         const int nblk = it.b1 - it.b0;
         const int last_blk = (len + kDecBN - 1) / kDecBN - 1;       // the block of the sequence with a ragged end
         if (warp == 1) {
             if (lane == 0) {
-                bool ok = true;
-                mbar_arrive_expect_tx(bar_q, (uint32_t)(KCH * q_box_heads * 128));
-                for (int c = 0; c < KCH; ++c) tma_load_3d(sQ + c * kChunkBytes, &mapQ, bar_q, c * 64, it.kvh * p.G, it.s);
-                mbar_arrive_expect_tx(bar_k, L::kTileBytes);
-                for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, it.kvh, seq_a + it.b0 * kDecBN);
-                mbar_arrive_expect_tx(bar_v, L::kTileBytes);
-                for (int c = 0; c < KCH; ++c) tma_load_3d(sV + c * kChunkBytes, &mapV, bar_v, c * 64, it.kvh, seq_a + it.b0 * kDecBN);
-                auto issue_s = [&]() {
+                bool ok = prod_ok && mbar_wait(bar_q, items_done & 1, kDecWaitCycles);
+                for (int j = 0; j < nblk && ok; ++j) {
+                    const uint32_t g = g0 + j, b = g & 1;
+                    // S_g goes where S_{g-2} and P_{g-2} were: PV_{g-2} is in front of it in issue order
+                    if (g >= 2) ok = confirm_s(g - 2);
+                    ok = ok && wait_full(2 * g);
+                    if (!ok) break;
+                    const uint32_t sK = sRing + ((2 * g) % kDecRing) * L::kTileBytes;
                     tc_fence_after();
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint32_t off = (kk >> 2) * kChunkBytes + (kk & 3) * 32;
-                        mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), idesc_s, kk > 0);
+                        mma_ss(tmem + b * 128, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), idesc_s, kk > 0);
                     }
-                    tc_commit(bar_s);
-                };
-                ok = mbar_wait(bar_q, items_done & 1, kDecWaitCycles) && mbar_wait(bar_k, blk0 & 1, kDecWaitCycles);
-                if (ok) issue_s();
-                for (int j = 0; j < nblk && ok; ++j) {
-                    const uint32_t ph = (blk0 + j) & 1;
-                    ok = mbar_wait(bar_s, ph, kDecWaitCycles);               // S_j done: the K buffer is free
-                    if (!ok) break;
-                    if (j + 1 < nblk) {
-                        mbar_arrive_expect_tx(bar_k, L::kTileBytes);
-                        for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, it.kvh, seq_a + (it.b0 + j + 1) * kDecBN);
-                    }
-                    ok = mbar_wait(bar_p0, ph, kDecWaitCycles) && mbar_wait(bar_v, ph, kDecWaitCycles);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int kk = 0; kk < kDecBN / 32; ++kk)
-                        mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
-                    ok = mbar_wait(bar_p1, ph, kDecWaitCycles);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int kk = kDecBN / 32; kk < kDecBN / 16; ++kk)
-                        mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, 1);
-                    tc_commit(bar_o);
-                    if (j + 1 < nblk) {
-                        ok = mbar_wait(bar_k, (blk0 + j + 1) & 1, kDecWaitCycles);
-                        if (!ok) break;
-                        issue_s();                                         // in issue order behind PV_j, which reads P_j from the same columns
-                    }
-                    ok = mbar_wait(bar_o, ph, kDecWaitCycles);              // PV_j done: the V buffer is free
-                    if (!ok) break;
-                    if (j + 1 < nblk) {
-                        mbar_arrive_expect_tx(bar_v, L::kTileBytes);
-                        for (int c = 0; c < KCH; ++c) tma_load_3d(sV + c * kChunkBytes, &mapV, bar_v, c * 64, it.kvh, seq_a + (it.b0 + j + 1) * kDecBN);
-                    }
+                    tc_commit(bar_s + 8 * b);
+                    s_issued = g + 1;
+                    if (j > 0) ok = issue_pv(g - 1, j > 1);
+                    ok = ok && pump();
                 }
-                if (!ok) { *abort_gen = 1; atomicExch(p.status, DASH_ERR_TIMEOUT); }
+                if (ok) ok = issue_pv(g0 + nblk - 1, nblk > 1);
+                // the item's last S is complete: the Q tile may take the next item's rows while this item's O is read out and merged
+                if (ok) ok = confirm_s(g0 + nblk - 1);
+                const int next = item + (int)gridDim.x;
+                if (ok && next < n_items) issue_q(get_item(next));
+                if (ok) ok = pump();
+                if (!ok) { prod_ok = false; *abort_gen = 1; atomicExch(p.status, DASH_ERR_TIMEOUT); }
             }
-        } else {
+            __syncwarp();
+        } else if (warp == 0) {
             // ---- softmax warp.  Only rows 0..G-1 of the 128-row tile exist, so the scores are fetched in the 16-row shape
             // (tcgen05.ld.16x256b): thread t holds, of row t / 4, the keys 8u + 2 (t % 4) + {0, 1} of every group u of 8 keys
             // (and the same of row t / 4 + 8, which is not a real head and is ignored).  Four threads share a row: 32 exponentials
             // per thread and block instead of 128.  P goes back in the 16x128b shape, whose 32-bit column 4u + (t % 4) is exactly
             // the pair of keys the thread holds. ----
-            const int sub = lane & 3, hrow = lane >> 2;         // position within the row's four threads, row (query head of the group)
+            const int sub = lane & 3;                           // position within the row's four threads
             float m = -INFINITY, l = 0.f;                       // m: common to the row's threads, l: this thread's share
             bool ok = true;
             for (int j = 0; j < nblk; ++j) {
-                const uint32_t ph = (blk0 + j) & 1;
-                ok = mbar_wait(bar_s, ph, kDecWaitCycles);
+                const uint32_t g = g0 + j, b = g & 1, ph = (g >> 1) & 1;
+                const uint32_t tS = tmem + b * 128, tP = tS;
+                ok = mbar_wait(bar_s + 8 * b, ph, kDecWaitCycles);
                 if (!ok || *abort_gen) { ok = false; break; }
                 tc_fence_after();
                 uint32_t raw[64];
@@ -314,7 +437,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 const float msl = m_new * p.scale_log2;
                 const float alpha = grow ? ex2((m - m_new) * p.scale_log2) : 1.0f;
                 if (j > 0 && __any_sync(0xffffffffu, grow)) {
-                    ok = mbar_wait(bar_o, (blk0 + j - 1) & 1, kDecWaitCycles);
+                    ok = mbar_wait(bar_o + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, kDecWaitCycles);     // PV_{g-1} done
                     if (!ok) break;
                     tc_fence_after();
                     const float a_row = __shfl_sync(0xffffffffu, alpha, (lane * 4) & 31);   // lane r < 8 rescales row r of O
@@ -331,13 +454,14 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                 }
                 if (ragged) {
                     // cached rows past the end of the sequence may hold anything: zero them (0 * garbage must not make a NaN)
-                    ok = mbar_wait(bar_v, ph, kDecWaitCycles);
+                    ok = wait_full(2 * g + 1);
                     if (!ok) break;
+                    uint8_t* vt = smem_gen + L::kRing + ((2 * g + 1) % kDecRing) * L::kTileBytes;
                     for (int r = lane; r < kDecBN; r += 32) {
                         if (r >= valid) {
 #pragma unroll
                             for (int c = 0; c < KCH; ++c) {
-                                uint4* rowp = reinterpret_cast<uint4*>(smem_gen + L::kV + c * kChunkBytes + r * 128);
+                                uint4* rowp = reinterpret_cast<uint4*>(vt + c * kChunkBytes + r * 128);
 #pragma unroll
                                 for (int e = 0; e < 8; ++e) rowp[e] = make_uint4(0, 0, 0, 0);
                             }
@@ -363,20 +487,20 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     tmem_st16x128_x8(tP + half * 32, &pk[half * 16]);
                     tmem_wait_st();
                     tc_fence_before();
-                    mbar_arrive(half == 0 ? bar_p0 : bar_p1);
+                    mbar_arrive((half == 0 ? bar_p0 : bar_p1) + 8 * b);
                 }
                 l = l * alpha + (sum2.x + sum2.y);
                 m = m_new;
             }
-            if (ok) ok = mbar_wait(bar_o, (blk0 + nblk - 1) & 1, kDecWaitCycles);
+            const uint32_t gl = g0 + nblk - 1;
+            if (ok) ok = mbar_wait(bar_o + 8 * (gl & 1), (gl >> 1) & 1, kDecWaitCycles);
             // row sum: the four threads' shares; then lane r < G writes row r (its m and l sit in thread 4 r)
             l += __shfl_xor_sync(0xffffffffu, l, 1);
             l += __shfl_xor_sync(0xffffffffu, l, 2);
             const float m_row = __shfl_sync(0xffffffffu, m, (lane * 4) & 31), l_row = __shfl_sync(0xffffffffu, l, (lane * 4) & 31);
-            (void)hrow;
             if (ok && !*abort_gen) {
                 tc_fence_after();
-                float* dst = p.partial + ((size_t)item * kDecRows + lane) * (D + 2);
+                float* dst = p.partial + ((size_t)item * kDecRows + lane) * (D + 4);
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t o[32];
@@ -384,19 +508,35 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                     tmem_wait_ld();
                     if (lane < p.G) {
 #pragma unroll
-                        for (int e = 0; e < 32; e += 2)
-                            *reinterpret_cast<float2*>(dst + c * 32 + e) = make_float2(__uint_as_float(o[e]), __uint_as_float(o[e + 1]));
+                        for (int e = 0; e < 32; e += 4)
+                            *reinterpret_cast<float4*>(dst + c * 32 + e) =
+                                make_float4(__uint_as_float(o[e]), __uint_as_float(o[e + 1]), __uint_as_float(o[e + 2]), __uint_as_float(o[e + 3]));
                     }
                 }
                 if (lane < p.G) { dst[D] = m_row; dst[D + 1] = l_row; }
+                __threadfence();
             } else if (!ok && lane == 0) {
                 *abort_gen = 1;
                 atomicExch(p.status, DASH_ERR_TIMEOUT);
             }
         }
+        // ---- end of the item: the partial result is in memory; the CTA that completes the head group's last item merges ----
         tc_fence_before();
-        __syncthreads();                      // end of the item: O read out, every tile buffer free
-        blk0 += (uint32_t)nblk;
+        __syncthreads();
+        int first, per;
+        if (self_plan) { per = sp.per[it.s]; first = sp.first[it.s] + it.kvh * per; }
+        else { const int2 sg = p.seg[it.s * p.Hkv + it.kvh]; first = sg.x; per = sg.y; }
+        if (tid == 0) {
+            int last = 0;
+            if (!*abort_gen) {
+                last = (atomicAdd(p.counters + it.s * p.Hkv + it.kvh, 1u) == (unsigned int)(per - 1));
+                __threadfence();
+            }
+            *last_gen = last;
+        }
+        __syncthreads();
+        if (*last_gen) decode_merge<D>(p, s_w, it.s, it.kvh, first, per < kMergeMaxSplits ? per : kMergeMaxSplits);
+        g0 += (uint32_t)nblk;
         ++items_done;
     }
     tc_fence_before();
@@ -407,79 +547,19 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     }
 }
 
-// One CTA per (sequence, query head): combine the partial results of the key splits.  The weights of the splits are formed
-// in parallel over the splits; the sums over the splits run in kMergeGroups thread groups (each takes every kMergeGroups-th split,
-// independent loads, unrolled) that meet in shared memory.
-constexpr int kMergeMaxSplits = 1024, kMergeGroups = 4, kMergeThreads = 128 * kMergeGroups;
-template <bool OUT_F32>
-__global__ void __launch_bounds__(kMergeThreads)
-decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ seg, const int32_t* __restrict__ cu, int S, int target,
-                    int Hq, int G, int D, float scale_log2, float scale, void* __restrict__ out, int64_t ldo, float* __restrict__ lse) {
-    __shared__ float s_w[kMergeMaxSplits];
-    __shared__ float s_red[kMergeThreads / 32];
-    __shared__ float s_acc[kMergeGroups][128];
-    __shared__ float s_m, s_l;
-    pdl_launch_dependents();
-    pdl_wait();                              // started while the decode kernel drains: its partial results are complete from here on
-    const int s = blockIdx.x / Hq, h = blockIdx.x % Hq;
-    const int kvh = h / G, row = h % G, Hkv = Hq / G;
-    __shared__ SelfPlan sp;
-    if (!seg) self_plan_build(sp, cu, S, Hkv, target);
-    const int2 sg = seg ? seg[s * Hkv + kvh] : make_int2(sp.first[s] + kvh * sp.per[s], sp.per[s]);
-    const int cnt = sg.y < kMergeMaxSplits ? sg.y : kMergeMaxSplits;
-    const size_t stride = (size_t)kDecRows * (D + 2);
-    const float* base = partial + ((size_t)sg.x * kDecRows + row) * (D + 2);
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    constexpr int NW = kMergeThreads / 32;
-    float mx = -INFINITY;
-    for (int i = threadIdx.x; i < cnt; i += kMergeThreads) mx = fmaxf(mx, base[i * stride + D]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) s_red[w] = mx;
-    __syncthreads();
-    if (threadIdx.x == 0) { float v = s_red[0]; for (int i = 1; i < NW; ++i) v = fmaxf(v, s_red[i]); s_m = v; }
-    __syncthreads();
-    const float mall = s_m;
-    float ls = 0.f;
-    for (int i = threadIdx.x; i < cnt; i += kMergeThreads) {
-        const float wi = exp2f((base[i * stride + D] - mall) * scale_log2);
-        s_w[i] = wi;
-        ls += wi * base[i * stride + D + 1];
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
-    __syncthreads();
-    if (lane == 0) s_red[w] = ls;
-    __syncthreads();
-    if (threadIdx.x == 0) { float v = 0.f; for (int i = 0; i < NW; ++i) v += s_red[i]; s_l = v; }
-    __syncthreads();
-    const float lall = s_l;
-    const int grp = threadIdx.x >> 7, c = threadIdx.x & 127;       // D <= 128: one column per thread of a group
-    float acc = 0.f;
-    if (c < D) {
-#pragma unroll 8
-        for (int i = grp; i < cnt; i += kMergeGroups) acc += s_w[i] * base[i * stride + c];
-    }
-    s_acc[grp][c] = acc;
-    __syncthreads();
-    if (grp == 0 && c < D) {
-        float v = 0.f;
-#pragma unroll
-        for (int gI = 0; gI < kMergeGroups; ++gI) v += s_acc[gI][c];
-        v = cnt > 0 ? v / lall : 0.f;
-        if (OUT_F32) reinterpret_cast<float*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = v;
-        else reinterpret_cast<__nv_bfloat16*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = __float2bfloat16(v);
-    }
-    if (lse && threadIdx.x == 0) lse[(int64_t)s * Hq + h] = cnt > 0 ? mall * scale + logf(lall) : -INFINITY;
+static int decode_grid() { return sm_count(); }
+static int decode_target(bool self_plan) {               // items aimed at: two per CTA when the CTAs plan (they go down to one each where that
+    const int t = (self_plan ? 2 : 4) * decode_grid();   // keeps them all busy), four per CTA with a plan kernel
+    return t < kMergeMaxSplits - 8 ? t : kMergeMaxSplits - 8;
 }
-
-static int decode_max_items(int S, int Hkv) { return 4 * sm_count() + S * Hkv; }
+static int decode_max_items(int S, int Hkv) { return 4 * decode_grid() + S * Hkv; }
 
 size_t decode_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D) {
     (void)n; (void)Hq;
     const size_t items = (size_t)decode_max_items(S, Hkv);
-    return 256 + align_up(items * sizeof(DecItem), 256) + align_up((size_t)S * Hkv * sizeof(int2), 256) + align_up((size_t)S * sizeof(int), 256) +
-           align_up(items * kDecRows * (size_t)(D + 2) * sizeof(float), 256);
+    return 256 + align_up((size_t)S * Hkv * sizeof(unsigned int), 256) + align_up(items * sizeof(DecItem), 256) +
+           align_up((size_t)S * Hkv * sizeof(int2), 256) + align_up((size_t)S * sizeof(int), 256) +
+           align_up(items * kDecRows * (size_t)(D + 4) * sizeof(float), 256);
 }
 
 // bf16 tensor [rows, heads, D]: box = 64 x box_heads x box_rows, 128-byte swizzle
@@ -529,39 +609,43 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
     if (!(scale > 0.f)) return DASH_ERR_INVALID_ARG;
     if (!ws || ((uintptr_t)ws % 256) || ws_bytes < decode_ws_bytes(n, S, Hq, Hkv, D)) return DASH_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    if (n == 0) {                             // no cached key anywhere: zeros and -inf
+        decode_empty_kernel<<<S, 128, 0, st>>>(Hq, D, out, ldo, lse);
+        DASH_CUDA_TRY(cudaGetLastError());
+        return DASH_OK;
+    }
     const int max_items = decode_max_items(S, Hkv);
     char* w = (char*)ws;
-    DecItem* plan = (DecItem*)(w + 256);
-    int2* seg = (int2*)(w + 256 + align_up((size_t)max_items * sizeof(DecItem), 256));
+    unsigned int* counters = (unsigned int*)(w + 256);
+    DecItem* plan = (DecItem*)((char*)counters + align_up((size_t)S * Hkv * sizeof(unsigned int), 256));
+    int2* seg = (int2*)((char*)plan + align_up((size_t)max_items * sizeof(DecItem), 256));
     int* seq_first = (int*)((char*)seg + align_up((size_t)S * Hkv * sizeof(int2), 256));
     float* partial = (float*)((char*)seq_first + align_up((size_t)S * sizeof(int), 256));
     const bool self_plan = S <= kSelfPlanSeqs;
-    const int target = 4 * sm_count();        // items aimed at: four per SM (self-planning CTAs go down to one item each where that keeps them all busy)
-    if (!self_plan) {
-        decode_plan_kernel<<<1, 256, 0, st>>>(cu_seqlens, S, Hkv, target, plan, seg, (int*)(w + 4), (unsigned int*)w, max_items, seq_first);
+    const int target = decode_target(self_plan);
+    if (self_plan) {
+        DASH_CUDA_TRY(cudaMemsetAsync(counters, 0, (size_t)S * Hkv * sizeof(unsigned int), st));
+    } else {
+        decode_plan_kernel<<<1, 256, 0, st>>>(cu_seqlens, S, Hkv, target, plan, seg, (int*)(w + 4), counters, max_items, seq_first);
         DASH_CUDA_TRY(cudaGetLastError());
     }
-    const float scale_log2 = scale * 1.4426950408889634f;
-    if (n > 0) {
-        CUtensorMap mq, mk, mv;
-        int rc;
-        const int box_heads = Hq < kDecRows ? Hq : kDecRows;
-        if ((rc = make_map_heads_box(&mq, q, S, Hq, D, ldq, box_heads, 1)) != DASH_OK) return rc;
-        if ((rc = make_map_heads_box(&mk, Kc, n, Hkv, D, ldk, 1, kDecBN)) != DASH_OK) return rc;
-        if ((rc = make_map_heads_box(&mv, Vc, n, Hkv, D, ldv, 1, kDecBN)) != DASH_OK) return rc;
-        DecParams p;
-        p.cu = cu_seqlens; p.S = S; p.Hq = Hq; p.Hkv = Hkv; p.G = G;
-        p.scale = scale; p.scale_log2 = scale_log2;
-        p.partial = partial; p.plan = self_plan ? nullptr : plan; p.n_items = (const int*)(w + 4); p.ticket = (unsigned int*)w;
-        p.target = target;
-        p.status = status_word_ptr();
-        if (!p.status) return DASH_ERR_CUDA;
-        int grid = 2 * sm_count();
-        if (grid > max_items) grid = max_items;
-        rc = D == 128 ? launch_decode<128>(mq, mk, mv, p, box_heads, grid, st) : launch_decode<64>(mq, mk, mv, p, box_heads, grid, st);
-        if (rc != DASH_OK) return rc;
-    }
-    DASH_CUDA_TRY(launch_pdl(decode_merge_kernel<false>, S * Hq, kMergeThreads, 0, st, (const float*)partial, (const int2*)(self_plan ? nullptr : seg),
-                             cu_seqlens, S, target, Hq, G, D, scale_log2, scale, out, ldo, lse));
-    return DASH_OK;
+    CUtensorMap mq, mk, mv;
+    int rc;
+    const int box_heads = Hq < kDecRows ? Hq : kDecRows;
+    if ((rc = make_map_heads_box(&mq, q, S, Hq, D, ldq, box_heads, 1)) != DASH_OK) return rc;
+    if ((rc = make_map_heads_box(&mk, Kc, n, Hkv, D, ldk, 1, kDecBN)) != DASH_OK) return rc;
+    if ((rc = make_map_heads_box(&mv, Vc, n, Hkv, D, ldv, 1, kDecBN)) != DASH_OK) return rc;
+    DecParams p;
+    p.cu = cu_seqlens; p.S = S; p.Hq = Hq; p.Hkv = Hkv; p.G = G;
+    p.scale = scale; p.scale_log2 = scale * 1.4426950408889634f;
+    p.partial = partial; p.plan = self_plan ? nullptr : plan; p.seg = seg; p.n_items = (const int*)(w + 4); p.counters = counters;
+    p.target = target;
+    p.status = status_word_ptr();
+    if (!p.status) return DASH_ERR_CUDA;
+    p.out = out; p.ldo = ldo; p.lse = lse;
+    int grid = decode_grid();
+    const int64_t most = (n / kDecBN + S) * Hkv;          // no plan has more items than this
+    if (grid > most) grid = (int)most;
+    if (grid > max_items) grid = max_items;
+    return D == 128 ? launch_decode<128>(mq, mk, mv, p, box_heads, grid, st) : launch_decode<64>(mq, mk, mv, p, box_heads, grid, st);
 }
