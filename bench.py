@@ -614,7 +614,7 @@ def setup_decode(args, dash, dev, rank):
     t_full = timer_simple(lambda: attn_over(False), 5)
     t_halt = timer_simple(lambda: attn_over(True), 5)
 
-    # the same 28 calls replayed as one CUDA graph: what the GPU needs once the host no longer issues the 28 memsets and 28 launches one by one
+    # the same 28 calls replayed as one CUDA graph: what the GPU needs once the host no longer issues the 56 launches one by one
     # (at short caches the eager loop is bound by the host's launch rate)
     def graphed(halting):
         try:
@@ -648,15 +648,20 @@ def setup_decode(args, dash, dev, rank):
              "speedup_measured": t_full / t_halt,
              "dense_decode_attention_graph_ms": t_full_g, "halted_decode_attention_graph_ms": t_halt_g,
              "speedup_measured_graph": (t_full_g / t_halt_g) if t_full_g and t_halt_g else None,
+             # one call on one dense cache as it runs inside the graph (the 28 dense caches are equally long): what the GPU needs per call
+             # once the host's issue time is out of the way; the roofline object below times one call issued eagerly behind an L2 flush
+             "dense_call_in_graph_us": (t_full_g / Lr * 1e3) if t_full_g else None,
+             "dense_call_in_graph_GBps": (T * row_b / (t_full_g / Lr * 1e-3) / 1e9) if t_full_g else None,
+             "dense_call_in_graph_frac_of_hbm_peak": (T * row_b / (t_full_g / Lr * 1e-3) / 1e9 / measured_peaks()["hbm_gbs"]) if t_full_g else None,
              "value_counts": "new tokens per second of the attention part of one decoding step over all 28 caches (batch 1)"}
     return {
         "workload": f"decoding stage after a halted prefill of {T} tokens: attention of one new token over the KV caches of {Lr} "
                     f"Qwen2.5-7B-shaped blocks ({l_s} with {T} cached tokens, {Lr - l_s} with {K}), bf16, batch 1",
-        "dtype": "bf16", "step": (lambda: attn_over(True)), "h2d": h2d, "d2h": d2h, "tokens": 1, "launches": Lr,
-        "launch_note": f"{Lr} x decode kernel (each behind a memset of its arrival counters; the merge of the key splits runs inside it)",
+        "dtype": "bf16", "step": (lambda: attn_over(True)), "h2d": h2d, "d2h": d2h, "tokens": 1, "launches": 2 * Lr,
+        "launch_note": f"{Lr} x (decode kernel, merge kernel)",
         "h2d_bytes": _bytes(q_host), "d2h_bytes": _bytes(out_h), "extra": extra,
         "attn": (lambda: dash.dash_decode_attention(q, Kc, Vc, cu_full, out=out, ws=ws)), "attn_flops": 4.0 * sh.Hq * sh.D * T,
-        "attn_bytes": float(T * row_b), "attn_name": f"decode_kernel<{sh.D}> (key splits merged by the last CTA to arrive) over {T} cached tokens (HBM-bound: K and V read once)",
+        "attn_bytes": float(T * row_b), "attn_name": f"decode_kernel<{sh.D}> + merge over {T} cached tokens (HBM-bound: K and V read once)",
         "norm": (lambda: dash.dash_delta_norm(U, Hh, r_out=r, Hres_out=Ht, tau=0.0, cu_seqlens=cu_full, mask_out=mask)), "norm_bytes": T * (3 * sh.d * 2 + 5),
         "compact": (lambda: dash.dash_compact(mask2, cu_full, rows=[Ht], rows_out=[Hn], pos_in=pos, tok_in=pos, want_idx=False, ws=cws, outputs=oo)),
         "compact_bytes": k2 * (2 * sh.d * 2 + 16) + T * 9, "compact_rows": k2, "row_bytes": sh.d * 2,
