@@ -167,7 +167,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base + L::kQ, sK = smem_base + L::kK, sV = smem_base + L::kV;
     const uint32_t bars = smem_base + L::kBars;
-    const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_o = bars + 32, bar_p0 = bars + 40, bar_p1 = bars + 48;
+    const uint32_t bar_q = bars, bar_k = bars + 8, bar_v = bars + 16, bar_s = bars + 24, bar_o = bars + 32, bar_p0 = bars + 40, bar_p1 = bars + 48, bar_o0 = bars + 56;
     const uint32_t tmem_slot = bars + 64;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot_gen = reinterpret_cast<volatile uint32_t*>(smem_gen + L::kBars + 64);
@@ -180,7 +180,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     if (warp == 4) {
         if (lane == 0) {
             mbar_init(bar_q, 1); mbar_init(bar_k, 1); mbar_init(bar_v, 1);
-            mbar_init(bar_s, 1); mbar_init(bar_o, 1); mbar_init(bar_p0, 128); mbar_init(bar_p1, 128);
+            mbar_init(bar_s, 1); mbar_init(bar_o, 1); mbar_init(bar_o0, 1); mbar_init(bar_p0, 128); mbar_init(bar_p1, 128);
             *abort_gen = 0;
             fence_barrier_init();
             fence_proxy_async_smem();
@@ -268,6 +268,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
                 for (int kk = 0; kk < kBN / 32; ++kk)
                     mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
+                tc_commit(bar_o0);
             }
             ok = all_ok(mbar_wait(bar_p1, ph, kWaitCycles));
             if (!ok) break;
@@ -328,6 +329,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
                 for (int kk = 0; kk < kBN / 32; ++kk)
                     mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
+                tc_commit(bar_o0);                            // for a softmax thread that has to rescale O in the middle of the block
                 ok = mbar_wait(bar_p1, ph, kWaitCycles);
                 if (!ok) break;
                 tc_fence_after();
@@ -369,47 +371,27 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_base + c * 32, &sreg[c * 32]);
             tmem_wait_ld();
             const bool diag = (j == qt);
-            if (diag) {
+            auto mask_diag = [&](int c0, int c1) {
 #pragma unroll
-                for (int c = 0; c < 128; ++c)
+                for (int c = c0; c < c1; ++c)
                     if (c > row) sreg[c] = 0xff800000u;     // -inf: keys after the query (and past the sequence end)
-            }
-            // four independent chains of three-input max keep the reduction short and off the latency-bound path
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+            };
+            if (diag) mask_diag(0, 128);
+            // The reference m of the row (exponentials are taken of s - m) is the first block's row maximum and stays unless a later
+            // block towers over it: a block's exponentials are formed against the m at hand without looking for the block's maximum,
+            // and their sum tells whether that was safe.  Sums below 2^64 are (P up to 2^64 is exact in bf16's range and harmless in
+            // the fp32 sums of P V and l); a larger or non-finite sum sends the warp through the rescaling path below.
+            if (j == 0) {
+                // four independent chains of three-input max keep the reduction short and off the latency-bound path
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 128; c += 8) {
-                mx0 = fmax3(mx0, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
-                mx1 = fmax3(mx1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
-                mx2 = fmax3(mx2, __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
-                mx3 = fmax3(mx3, __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
-            }
-            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            // Lazy rescale: the reference max m only moves when the block max exceeds it by more than
-            // 2^8 in the exponent; until then P is formed against the old m (values up to 256, safe in
-            // bf16 / fp32) and O needs no correction.
-            const bool grow = (mx - m) * p.scale_log2 > 8.0f;
-            const float m_new = grow ? mx : m;
-            const float msl = m_new * p.scale_log2;
-            const float alpha = grow ? ex2((m - m_new) * p.scale_log2) : 1.0f;
-            if (j > 0) {
-                // O still holds the previous blocks' sum scaled by the old reference max
-                const bool need = __any_sync(0xffffffffu, grow);
-                if (need) {
-                    ok = mbar_wait(bar_o, (blk0 + j - 1) & 1, kWaitCycles);
-                    if (!ok) break;
-                    tc_fence_after();
-                    // rare path (the reference max moves in the first blocks only): small chunks, not
-                    // unrolled, so it adds no register pressure to the hot loop around it
-#pragma unroll 1
-                    for (int c = 0; c < D / 8; ++c) {
-                        uint32_t o[8];
-                        tmem_ld8(tO + lane_base + c * 8, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        tmem_st8(tO + lane_base + c * 8, o);
-                    }
+                for (int c = 0; c < 128; c += 8) {
+                    mx0 = fmax3(mx0, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+                    mx2 = fmax3(mx2, __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
+                    mx3 = fmax3(mx3, __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
                 }
+                m = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));          // finite: key 0 is visible to every query row
             }
             if (diag) {
                 // keys past the end of the sequence: their V rows may hold anything (another
@@ -426,33 +408,76 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     fence_proxy_async_smem();
                 }
             }
-            // scale-subtract and row sums on packed fp32 pairs (two lanes per FMA-pipe instruction)
-            float2 sumA = make_float2(0.f, 0.f), sumB = make_float2(0.f, 0.f);
-            const float2 sl2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-msl, -msl);
+            const float2 sl2 = make_float2(p.scale_log2, p.scale_log2);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
+                // scale-subtract and row sums on packed fp32 pairs (two lanes per FMA-pipe instruction); P is packed in place
+                auto exps = [&]() -> float {
+                    float2 sumA = make_float2(0.f, 0.f), sumB = make_float2(0.f, 0.f);
+                    const float msl = m * p.scale_log2;
+                    const float2 nm2 = make_float2(-msl, -msl);
 #pragma unroll
-                for (int c = half * 64; c < half * 64 + 64; c += 4) {
-                    const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), sl2, nm2);
-                    const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), sl2, nm2);
-                    float2 pa, pb;
-                    pa.x = ex2(xa.x);
-                    pa.y = (kExpPolyPer4 >= 2) ? ex2_poly(xa.y) : ex2(xa.y);
-                    pb.x = ex2(xb.x);
-                    pb.y = (kExpPolyPer4 >= 1) ? ex2_poly(xb.y) : ex2(xb.y);
-                    sumA = __fadd2_rn(sumA, pa);
-                    sumB = __fadd2_rn(sumB, pb);
-                    sreg[c >> 1] = pack_bf16(pa.x, pa.y);
-                    sreg[(c >> 1) + 1] = pack_bf16(pb.x, pb.y);
+                    for (int c = half * 64; c < half * 64 + 64; c += 4) {
+                        const float2 xa = __ffma2_rn(make_float2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), sl2, nm2);
+                        const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), sl2, nm2);
+                        float2 pa, pb;
+                        pa.x = ex2(xa.x);
+                        pa.y = (kExpPolyPer4 >= 2) ? ex2_poly(xa.y) : ex2(xa.y);
+                        pb.x = ex2(xb.x);
+                        pb.y = (kExpPolyPer4 >= 1) ? ex2_poly(xb.y) : ex2(xb.y);
+                        sumA = __fadd2_rn(sumA, pa);
+                        sumB = __fadd2_rn(sumB, pb);
+                        sreg[c >> 1] = pack_bf16(pa.x, pa.y);
+                        sreg[(c >> 1) + 1] = pack_bf16(pb.x, pb.y);
+                    }
+                    return (sumA.x + sumA.y) + (sumB.x + sumB.y);
+                };
+                float hs = exps();
+                if (__any_sync(0xffffffffu, row_valid && !(hs < 1.8446744e19f))) {     // (rows past the sequence's end may hold anything and are never written)
+                    // rare: some row of the warp met scores far above its reference.  The half's scores are still in TMEM (P has not
+                    // been stored over them): fetch them again, move m where the half's maximum asks for it (the rows that need not
+                    // move keep theirs), bring O and l to the new m -- O once every product issued so far has landed -- and redo.
+                    tmem_ld32(tS + lane_base + half * 64, &sreg[half * 64]);
+                    tmem_ld32(tS + lane_base + half * 64 + 32, &sreg[half * 64 + 32]);
+                    tmem_wait_ld();
+                    if (diag) mask_diag(half * 64, half * 64 + 64);
+                    float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+                    for (int c = half * 64; c < half * 64 + 64; c += 4) {
+                        mx0 = fmax3(mx0, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
+                        mx1 = fmax3(mx1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+                    }
+                    const float mx = fmaxf(mx0, mx1);
+                    const bool grow = (mx - m) * p.scale_log2 > 8.0f;
+                    const float m_new = grow ? mx : m;
+                    const float alpha = grow ? ex2((m - m_new) * p.scale_log2) : 1.0f;
+                    if (half == 1) ok = mbar_wait(bar_o0, ph, kWaitCycles);                       // the first half's products of this block
+                    else if (j > 0) ok = mbar_wait(bar_o, (blk0 + j - 1) & 1, kWaitCycles);       // the blocks before
+                    if (!ok) break;
+                    if (half == 1 || j > 0) {
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int c = 0; c < D / 8; ++c) {
+                            uint32_t o[8];
+                            tmem_ld8(tO + lane_base + c * 8, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st8(tO + lane_base + c * 8, o);
+                        }
+                    }
+                    l *= alpha;
+                    m = m_new;
+                    hs = exps();
                 }
                 // the first 64 keys of P go out (and their PV steps start) while the rest is still being formed
                 tmem_st32(tP + lane_base + half * 32, &sreg[half * 32]);
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(half == 0 ? bar_p0 : bar_p1);
+                l += hs;
             }
-            l = l * alpha + ((sumA.x + sumA.y) + (sumB.x + sumB.y));
-            m = m_new;
+            if (!ok) break;
         }
         if (ok) ok = mbar_wait(bar_o, (blk0 + nblk - 1) & 1, kWaitCycles);
         if (ok && !*abort_gen) {

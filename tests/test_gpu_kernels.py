@@ -257,13 +257,17 @@ def test_compact_empty_input():
 
 
 # ------------------------------------------------------------------ step 4
-def _attention_case(lengths, Hq, Hkv, D, dtype, seed, rows=None, pad=0, tol=TOL):
+def _attention_case(lengths, Hq, Hkv, D, dtype, seed, rows=None, pad=0, tol=TOL, key_gain=None):
     cu = wl.cu_from_lengths(lengths)
     n = int(cu[-1])
     g = torch.Generator().manual_seed(seed)
     Q = torch.randn(n + pad, Hq, D, generator=g).to(dtype)
     K = torch.randn(n + pad, Hkv, D, generator=g).to(dtype)
     V = torch.randn(n + pad, Hkv, D, generator=g).to(dtype)
+    if key_gain is not None:     # keys from position `at` of every sequence on are `gain` times longer
+        pos = wl.positions(cu).long()
+        for at, gain in key_gain:
+            K[:n][pos >= at] *= gain
     if pad:          # rows past the packed end hold poison that must never reach an output
         Q[n:], K[n:], V[n:] = float("nan"), float("inf"), float("nan")
     O, lse = dash.dash_varlen_attention(Q.to(DEV), K.to(DEV), V.to(DEV), cu.to(DEV), max(lengths), want_lse=True)
@@ -364,6 +368,14 @@ def test_attention_ragged_multi_tile_gqa():
 
 def test_attention_varlen_with_empty_and_short_sequences_and_poisoned_tail():
     _attention_case([129, 0, 1, 515, 64], 14, 2, 128, torch.bfloat16, 3, pad=200)
+
+
+def test_attention_scores_that_tower_over_the_first_key_block():
+    # The kernel keeps the first key block's row maximum as the reference of the exponentials and only moves it when a block's
+    # sum says it must.  Here later keys are 40, then 100 times longer: scores tens of units above everything before them, the
+    # jumps falling into the second half of a block (position 200), the first half (position 650) and a block's first key (1024).
+    _attention_case([1500, 700], 4, 2, 128, torch.bfloat16, 21, key_gain=[(200, 40.0), (650, 2.5), (1024, 3.0)])
+    _attention_case([900], 2, 1, 64, torch.bfloat16, 22, key_gain=[(130, 60.0)], pad=4)
 
 
 def test_attention_head_dim_64_fp32():
