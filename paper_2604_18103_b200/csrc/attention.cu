@@ -72,11 +72,6 @@ constexpr int kBN = 128;                 // keys per block
 constexpr int kAttnThreads = 160;
 constexpr long long kWaitCycles = 4000000000LL;   // ~2 s: a wait that long is reported, not retried
 constexpr uint32_t kTmemCols = 256;
-// how many of every four exponentials are evaluated on the FMA pipe instead of the MUFU
-#ifndef DASH_EXP_POLY_PER4
-#define DASH_EXP_POLY_PER4 0
-#endif
-constexpr int kExpPolyPer4 = DASH_EXP_POLY_PER4;
 
 struct AttnParams {
     const int32_t* cu;
@@ -422,9 +417,9 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                         const float2 xb = __ffma2_rn(make_float2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), sl2, nm2);
                         float2 pa, pb;
                         pa.x = ex2(xa.x);
-                        pa.y = (kExpPolyPer4 >= 2) ? ex2_poly(xa.y) : ex2(xa.y);
+                        pa.y = ex2(xa.y);
                         pb.x = ex2(xb.x);
-                        pb.y = (kExpPolyPer4 >= 1) ? ex2_poly(xb.y) : ex2(xb.y);
+                        pb.y = ex2(xb.y);
                         sumA = __fadd2_rn(sumA, pa);
                         sumB = __fadd2_rn(sumB, pb);
                         sreg[c >> 1] = pack_bf16(pa.x, pa.y);

@@ -201,20 +201,6 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return d;
 }
 
-// 2^x on the FMA pipe (no MUFU), for x <= 2^21: split x = floor(x) + f with a round-down add of
-// 1.5 * 2^23 (the integer lands in the low mantissa bits), evaluate a cubic fit of 2^f on [0,1)
-// (max relative error 8.7e-5, far below the bf16 rounding applied to P afterwards) and add
-// floor(x) to the exponent field.  Inputs below -126 flush to 2^-126.
-__device__ __forceinline__ float ex2_poly(float x) {
-    x = fmaxf(x, -126.0f);
-    const float u = __fadd_rd(x, 12582912.0f);
-    const float f = x - (u - 12582912.0f);
-    float p = fmaf(f, 0.07707636058330536f, 0.2276366949081421f);
-    p = fmaf(p, f, 0.6951168775558472f);
-    p = fmaf(p, f, 1.0f);
-    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(u) << 23));
-}
-
 }  // namespace ptx
 
 // ---- host: tensor-map encoding through the driver entry point (no -lcuda) -----
