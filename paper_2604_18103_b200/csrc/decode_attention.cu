@@ -3,7 +3,7 @@
 // HBM-bound: every cached key/value row is read once.  The G = Hq / Hkv query heads that share one KV
 // head form the (mostly empty) 128-row operand of the tcgen05 MMAs, so K and V tiles stream through
 // shared memory once per KV head; the keys of a sequence are split over persistent CTAs (flash-decoding),
-// whose partial (max, sum, O) results a small merge kernel combines.
+// whose partial (max, sum, O) results a merge kernel spread over all SMs combines.
 //   plan kernel   : items (sequence, KV head, key-block range), sized so that one item exists per CTA (batches of up to 32 sequences: the CTAs plan for themselves) or four per SM (handed out by ticket)
 //   decode kernel : per item  S = Q K_j^T -> masked online softmax (one warp: the rows that exist) -> O += P V_j
 //   merge kernel  : O = sum_i 2^((m_i - m) c) O_i / sum_i 2^((m_i - m) c) l_i
@@ -28,7 +28,9 @@ struct DecParams {
     const int32_t* cu;
     int S, Hq, Hkv, G;
     float scale_log2, scale;
-    float* partial;             // [item][kDecRows][D + 2]: unnormalised O row, then m, l
+    float* partial;             // [item][kDecRows][D]: unnormalised O rows
+    float2* ml;                 // [Hq][max_items]: their (m, l); the splits of one head lie next to each other
+    int max_items;
     const DecItem* plan;        // null: the CTAs plan for themselves (S <= kSelfPlanSeqs)
     const int* n_items;
     unsigned int* ticket;
@@ -376,7 +378,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
             (void)hrow;
             if (ok && !*abort_gen) {
                 tc_fence_after();
-                float* dst = p.partial + ((size_t)item * kDecRows + lane) * (D + 2);
+                float* dst = p.partial + ((size_t)item * kDecRows + lane) * D;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t o[32];
@@ -388,7 +390,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                             *reinterpret_cast<float2*>(dst + c * 32 + e) = make_float2(__uint_as_float(o[e]), __uint_as_float(o[e + 1]));
                     }
                 }
-                if (lane < p.G) { dst[D] = m_row; dst[D + 1] = l_row; }
+                if (lane < p.G) p.ml[(size_t)(it.kvh * p.G + lane) * p.max_items + item] = make_float2(m_row, l_row);
             } else if (!ok && lane == 0) {
                 *abort_gen = 1;
                 atomicExch(p.status, DASH_ERR_TIMEOUT);
@@ -407,70 +409,94 @@ decode_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     }
 }
 
-// One CTA per (sequence, query head): combine the partial results of the key splits.  The weights of the splits are formed
-// in parallel over the splits; the sums over the splits run in kMergeGroups thread groups (each takes every kMergeGroups-th split,
-// independent loads, unrolled) that meet in shared memory.
-constexpr int kMergeMaxSplits = 1024, kMergeGroups = 4, kMergeThreads = 128 * kMergeGroups;
-template <bool OUT_F32>
+// The merge of the key splits, spread over the whole machine.  A unit is 32 output columns of one (sequence, query head); it goes to a
+// group of K warps (K = 1, 2, 4 or 8: as many as there are warps per unit, so that few units with many splits and many units with
+// few splits both fill the SMs).  Every warp of the group loads the splits' (m, l) pairs, lane = split (they lie next to each other:
+// coalesced), and forms the common maximum, the splits' weights and the denominator; then it sums its share of the splits, lane =
+// column, with the weights handed round by shuffles.  All loads of a unit go out before the first is waited for; the group meets in
+// shared memory.
+constexpr int kMergeThreads = 256;
+struct MergeParams {
+    const float* partial; const float2* ml; int max_items;
+    const int2* seg;            // with a plan: first item and number of items of every (sequence, KV head); else the CTAs plan for themselves
+    const int32_t* cu; int S, target, Hq, Hkv, G;
+    float scale_log2, scale;
+    __nv_bfloat16* out; int64_t ldo; float* lse;
+};
+template <int D, int K>
+__device__ __forceinline__ void decode_merge_units(const MergeParams& p, const SelfPlan& sp, float (*s_acc)[32]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int NW = kMergeThreads / 32, CH = D / 32;
+    constexpr int B = 32, ML = B * K / 32;               // splits of one round: B per warp, their (m, l) in ML registers per lane
+    const int n_units = p.S * p.Hq * CH;
+    const int sub = warp % K;
+    const int n_groups = (int)gridDim.x * (NW / K), gid = (int)blockIdx.x * (NW / K) + warp / K;
+    const size_t stride = (size_t)kDecRows * D;
+    for (int u = gid; u < n_units; u += n_groups) {
+        const int ch = u % CH, hd = (u / CH) % p.Hq, s = u / (CH * p.Hq);
+        const int kvh = hd / p.G, row = hd % p.G;
+        int first, cnt;
+        if (!p.seg) { cnt = sp.per[s]; first = sp.first[s] + kvh * cnt; }
+        else { const int2 sg = p.seg[s * p.Hkv + kvh]; first = sg.x; cnt = sg.y; }
+        const float* base = p.partial + ((size_t)first * kDecRows + row) * D + ch * 32 + lane;
+        const float2* mlb = p.ml + (size_t)hd * p.max_items + first;
+        float dv[B];
+        float2 ml[ML];
+#pragma unroll
+        for (int b = 0; b < B; ++b) { const int i = sub + b * K; dv[b] = (i < cnt) ? __ldcg(base + i * stride) : 0.f; }
+#pragma unroll
+        for (int j = 0; j < ML; ++j) { const int i = lane + 32 * j; ml[j] = (i < cnt) ? __ldcg(mlb + i) : make_float2(-INFINITY, 0.f); }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < ML; ++j) mx = fmaxf(mx, ml[j].x);
+        for (int i = lane + 32 * ML; i < cnt; i += 32) mx = fmaxf(mx, __ldcg(mlb + i).x);          // more than B * K splits: further rounds
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float ls = 0.f;
+#pragma unroll
+        for (int j = 0; j < ML; ++j) {
+            ml[j].x = exp2f((ml[j].x - mx) * p.scale_log2);     // the split's weight (0 where there is no split)
+            ls = fmaf(ml[j].x, ml[j].y, ls);
+        }
+        for (int i = lane + 32 * ML; i < cnt; i += 32) { const float2 v = __ldcg(mlb + i); ls = fmaf(exp2f((v.x - mx) * p.scale_log2), v.y, ls); }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+        float acc = 0.f;
+#pragma unroll
+        for (int b = 0; b < B; ++b) acc = fmaf(__shfl_sync(0xffffffffu, ml[(b * K) / 32].x, (sub + b * K) & 31), dv[b], acc);
+        for (int i = sub + B * K; i < cnt; i += K) acc = fmaf(exp2f((__ldcg(mlb + i).x - mx) * p.scale_log2), __ldcg(base + i * stride), acc);
+        if (K > 1) {
+            s_acc[warp][lane] = acc;
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + warp / K), "n"(K * 32) : "memory");
+            if (sub == 0) {
+                acc = 0.f;
+#pragma unroll
+                for (int j = 0; j < K; ++j) acc += s_acc[warp + j][lane];
+            }
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + warp / K), "n"(K * 32) : "memory");
+        }
+        if (sub == 0) {
+            const float v = cnt > 0 ? acc / ls : 0.f;
+            p.out[(int64_t)s * p.ldo + (int64_t)hd * D + ch * 32 + lane] = __float2bfloat16(v);
+            if (p.lse && ch == 0 && lane == 0) p.lse[(int64_t)s * p.Hq + hd] = cnt > 0 ? mx * p.scale + logf(ls) : -INFINITY;
+        }
+    }
+}
+
+template <int D>
 __global__ void __launch_bounds__(kMergeThreads)
-decode_merge_kernel(const float* __restrict__ partial, const int2* __restrict__ seg, const int32_t* __restrict__ cu, int S, int target,
-                    int Hq, int G, int D, float scale_log2, float scale, void* __restrict__ out, int64_t ldo, float* __restrict__ lse) {
-    __shared__ float s_w[kMergeMaxSplits];
-    __shared__ float s_red[kMergeThreads / 32];
-    __shared__ float s_acc[kMergeGroups][128];
-    __shared__ float s_m, s_l;
+decode_merge_kernel(const MergeParams p) {
+    __shared__ SelfPlan sp;
+    __shared__ float s_acc[kMergeThreads / 32][32];
     pdl_launch_dependents();
     pdl_wait();                              // started while the decode kernel drains: its partial results are complete from here on
-    const int s = blockIdx.x / Hq, h = blockIdx.x % Hq;
-    const int kvh = h / G, row = h % G, Hkv = Hq / G;
-    __shared__ SelfPlan sp;
-    if (!seg) self_plan_build(sp, cu, S, Hkv, target);
-    const int2 sg = seg ? seg[s * Hkv + kvh] : make_int2(sp.first[s] + kvh * sp.per[s], sp.per[s]);
-    const int cnt = sg.y < kMergeMaxSplits ? sg.y : kMergeMaxSplits;
-    const size_t stride = (size_t)kDecRows * (D + 2);
-    const float* base = partial + ((size_t)sg.x * kDecRows + row) * (D + 2);
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    constexpr int NW = kMergeThreads / 32;
-    float mx = -INFINITY;
-    for (int i = threadIdx.x; i < cnt; i += kMergeThreads) mx = fmaxf(mx, base[i * stride + D]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) s_red[w] = mx;
-    __syncthreads();
-    if (threadIdx.x == 0) { float v = s_red[0]; for (int i = 1; i < NW; ++i) v = fmaxf(v, s_red[i]); s_m = v; }
-    __syncthreads();
-    const float mall = s_m;
-    float ls = 0.f;
-    for (int i = threadIdx.x; i < cnt; i += kMergeThreads) {
-        const float wi = exp2f((base[i * stride + D] - mall) * scale_log2);
-        s_w[i] = wi;
-        ls += wi * base[i * stride + D + 1];
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
-    __syncthreads();
-    if (lane == 0) s_red[w] = ls;
-    __syncthreads();
-    if (threadIdx.x == 0) { float v = 0.f; for (int i = 0; i < NW; ++i) v += s_red[i]; s_l = v; }
-    __syncthreads();
-    const float lall = s_l;
-    const int grp = threadIdx.x >> 7, c = threadIdx.x & 127;       // D <= 128: one column per thread of a group
-    float acc = 0.f;
-    if (c < D) {
-#pragma unroll 8
-        for (int i = grp; i < cnt; i += kMergeGroups) acc += s_w[i] * base[i * stride + c];
-    }
-    s_acc[grp][c] = acc;
-    __syncthreads();
-    if (grp == 0 && c < D) {
-        float v = 0.f;
-#pragma unroll
-        for (int gI = 0; gI < kMergeGroups; ++gI) v += s_acc[gI][c];
-        v = cnt > 0 ? v / lall : 0.f;
-        if (OUT_F32) reinterpret_cast<float*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = v;
-        else reinterpret_cast<__nv_bfloat16*>(out)[(int64_t)s * ldo + (int64_t)h * D + c] = __float2bfloat16(v);
-    }
-    if (lse && threadIdx.x == 0) lse[(int64_t)s * Hq + h] = cnt > 0 ? mall * scale + logf(lall) : -INFINITY;
+    if (!p.seg) self_plan_build(sp, p.cu, p.S, p.Hkv, p.target);
+    // warps per unit: as many as the machine has per unit, at most the CTA's eight
+    const long long n_units = (long long)p.S * p.Hq * (D / 32), warps = (long long)gridDim.x * (kMergeThreads / 32);
+    if (n_units * 16 <= warps) decode_merge_units<D, 8>(p, sp, s_acc);
+    else if (n_units * 8 <= warps) decode_merge_units<D, 4>(p, sp, s_acc);
+    else if (n_units * 4 <= warps) decode_merge_units<D, 2>(p, sp, s_acc);
+    else decode_merge_units<D, 1>(p, sp, s_acc);
 }
 
 static int decode_max_items(int S, int Hkv) { return 4 * sm_count() + S * Hkv; }
@@ -479,7 +505,7 @@ size_t decode_ws_bytes(int64_t n, int S, int Hq, int Hkv, int D) {
     (void)n; (void)Hq;
     const size_t items = (size_t)decode_max_items(S, Hkv);
     return 256 + align_up(items * sizeof(DecItem), 256) + align_up((size_t)S * Hkv * sizeof(int2), 256) + align_up((size_t)S * sizeof(int), 256) +
-           align_up(items * kDecRows * (size_t)(D + 2) * sizeof(float), 256);
+           align_up(items * kDecRows * (size_t)D * sizeof(float), 256) + align_up(items * (size_t)Hq * sizeof(float2), 256);
 }
 
 // bf16 tensor [rows, heads, D]: box = 64 x box_heads x box_rows, 128-byte swizzle
@@ -521,7 +547,7 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
     if (Hq % Hkv) return DASH_ERR_INVALID_ARG;
     const int G = Hq / Hkv;
     if (G > kDecRows) return DASH_ERR_UNSUPPORTED;
-    if (n > 0x7fffffffLL || S > 0x7fffffff / Hq) return DASH_ERR_INVALID_ARG;
+    if (n > 0x7fffffffLL || S > 0x7fffffff / (Hq * 4)) return DASH_ERR_INVALID_ARG;      // the merge counts its units in an int
     if (!q || !out || (n > 0 && (!Kc || !Vc))) return DASH_ERR_INVALID_ARG;
     if (ldq < (int64_t)Hq * D || ldo < (int64_t)Hq * D || ldk < (int64_t)Hkv * D || ldv < (int64_t)Hkv * D) return DASH_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(out) || (n > 0 && (!aligned16(Kc) || !aligned16(Vc)))) return DASH_ERR_INVALID_ARG;
@@ -535,6 +561,7 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
     int2* seg = (int2*)(w + 256 + align_up((size_t)max_items * sizeof(DecItem), 256));
     int* seq_first = (int*)((char*)seg + align_up((size_t)S * Hkv * sizeof(int2), 256));
     float* partial = (float*)((char*)seq_first + align_up((size_t)S * sizeof(int), 256));
+    float2* ml = (float2*)((char*)partial + align_up((size_t)max_items * kDecRows * D * sizeof(float), 256));
     const bool self_plan = S <= kSelfPlanSeqs;
     const int target = 4 * sm_count();        // items aimed at: four per SM (self-planning CTAs go down to one item each where that keeps them all busy)
     if (!self_plan) {
@@ -552,7 +579,7 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
         DecParams p;
         p.cu = cu_seqlens; p.S = S; p.Hq = Hq; p.Hkv = Hkv; p.G = G;
         p.scale = scale; p.scale_log2 = scale_log2;
-        p.partial = partial; p.plan = self_plan ? nullptr : plan; p.n_items = (const int*)(w + 4); p.ticket = (unsigned int*)w;
+        p.partial = partial; p.ml = ml; p.max_items = max_items; p.plan = self_plan ? nullptr : plan; p.n_items = (const int*)(w + 4); p.ticket = (unsigned int*)w;
         p.target = target;
         p.status = status_word_ptr();
         if (!p.status) return DASH_ERR_CUDA;
@@ -561,7 +588,17 @@ extern "C" int dash_decode_attention(const void* q, const void* Kc, const void* 
         rc = D == 128 ? launch_decode<128>(mq, mk, mv, p, box_heads, grid, st) : launch_decode<64>(mq, mk, mv, p, box_heads, grid, st);
         if (rc != DASH_OK) return rc;
     }
-    DASH_CUDA_TRY(launch_pdl(decode_merge_kernel<false>, S * Hq, kMergeThreads, 0, st, (const float*)partial, (const int2*)(self_plan ? nullptr : seg),
-                             cu_seqlens, S, target, Hq, G, D, scale_log2, scale, out, ldo, lse));
+    MergeParams mp;
+    mp.partial = partial; mp.ml = ml; mp.max_items = max_items; mp.seg = self_plan ? nullptr : seg;
+    mp.cu = cu_seqlens; mp.S = S; mp.target = target; mp.Hq = Hq; mp.Hkv = Hkv; mp.G = G;
+    mp.scale_log2 = scale_log2; mp.scale = scale;
+    mp.out = (__nv_bfloat16*)out; mp.ldo = ldo; mp.lse = lse;
+    // one warp per unit at least, never more CTAs than SMs
+    const long long units = (long long)S * Hq * (D / 32);
+    long long mgrid = (units * 8 + kMergeThreads / 32 - 1) / (kMergeThreads / 32);
+    if (mgrid > sm_count()) mgrid = sm_count();
+    if (mgrid < 1) mgrid = 1;
+    if (D == 128) DASH_CUDA_TRY(launch_pdl(decode_merge_kernel<128>, (int)mgrid, kMergeThreads, 0, st, mp));
+    else DASH_CUDA_TRY(launch_pdl(decode_merge_kernel<64>, (int)mgrid, kMergeThreads, 0, st, mp));
     return DASH_OK;
 }

@@ -376,6 +376,8 @@ def test_attention_scores_that_tower_over_the_first_key_block():
     # jumps falling into the second half of a block (position 200), the first half (position 650) and a block's first key (1024).
     _attention_case([1500, 700], 4, 2, 128, torch.bfloat16, 21, key_gain=[(200, 40.0), (650, 2.5), (1024, 3.0)])
     _attention_case([900], 2, 1, 64, torch.bfloat16, 22, key_gain=[(130, 60.0)], pad=4)
+    # and the other way round: the first block's keys are the long ones, everything behind them all but vanishes against the reference
+    _attention_case([700], 4, 2, 128, torch.bfloat16, 23, key_gain=[(0, 50.0), (128, 0.02)])
 
 
 def test_attention_head_dim_64_fp32():
