@@ -432,12 +432,18 @@ int gemm_bf16(GemmEpilogueKind kind, const void* A, int64_t lda, const void* W, 
 }
 
 int launch_row_prep(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const void* H, int64_t ldh, int d, float rms_eps,
-                    float* inv_rms, const int32_t* n_dev, cudaStream_t st) {
+                    float* inv_rms, const int32_t* n_dev, cudaStream_t st, bool beside_front) {
     RopeFreqs fr;
     for (int i = 0; i < D / 2; ++i) fr.inv_freq[i] = pow(rope_base, -2.0 * i / D);
     int64_t blocks = (n + 7) / 8, cap = (int64_t)sm_count() * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
+    // beside_front: the kernel in front in the stream is one whose output this kernel does not read and that was itself an ordinary
+    // launch (the block step's attention item list): launched to start beside it -- the kernel has no griddepcontrol.wait, and its
+    // inputs were complete before the kernel in front started.
+    if (beside_front)
+        return launch_pdl(row_prep_kernel, (int)blocks, 256, 0, st, pos, n, D / 2, fr, table, (const char*)H, ldh * 2, d * 2 / 16, 1.0f / d,
+                          rms_eps, inv_rms, n_dev) == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
     row_prep_kernel<<<(int)blocks, 256, 0, st>>>(pos, n, D / 2, fr, table, (const char*)H, ldh * 2, d * 2 / 16, 1.0f / d, rms_eps, inv_rms, n_dev);
     return cudaGetLastError() == cudaSuccess ? DASH_OK : DASH_ERR_CUDA;
 }

@@ -42,6 +42,6 @@ int launch_f32_to_bf16(const float* src, int64_t ld_src, void* dst, int64_t ld_d
 // per row: (cos, sin) of pos * base^(-2i/D) into table [n, D/2] (table null: not formed; pos null: the row number is the position);
 // with inv_rms non-null also 1 / sqrt(mean(H_row^2) + eps) (bf16 H, row stride ldh)
 int launch_row_prep(const int32_t* pos, int64_t n, int D, double rope_base, float2* table, const void* H, int64_t ldh, int d, float rms_eps,
-                    float* inv_rms, const int32_t* n_dev, cudaStream_t st);
+                    float* inv_rms, const int32_t* n_dev, cudaStream_t st, bool beside_front = false);
 
 }  // namespace dash

@@ -343,7 +343,7 @@ static int attention_to_O(const dash_layer_cfg* cfg, const void* H_in, const int
         if (cfg->rope_table) { e.rope_table = (const float2*)cfg->rope_table; e.rope_pos = pos_in; e.rope_len = cfg->rope_table_len; }
         if (!cfg->rope_table || !cfg->inv_rms_in) {
             rc = launch_row_prep(pos_in, n, D, cfg->rope_base, cfg->rope_table ? nullptr : W.rope_tab, H_in, d, d, cfg->rms_eps,
-                                 cfg->inv_rms_in ? nullptr : W.inv_rms, n_dev, st);
+                                 cfg->inv_rms_in ? nullptr : W.inv_rms, n_dev, st, true);      // beside the item list in front
             if (rc != DASH_OK) return rc;
         }
         e.row_scale = cfg->inv_rms_in ? cfg->inv_rms_in : W.inv_rms;
