@@ -9,7 +9,7 @@ one (what the oracle's cost allows: 2048 rows over 26214 keys are about 4e11 fp6
 drawn so that every 128-row query tile of every sequence holds at least one of them, with the
 first / last row of every sequence and both sides of the tile boundaries; the rest through
 properties that hold at any size.  Measured error ratios are collected in
-gpurun_out/parity_errors.json (see conftest.py)."""
+parity_errors.json in the session's record folder (see conftest.py)."""
 import math
 
 import numpy as np
