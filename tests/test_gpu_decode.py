@@ -49,6 +49,11 @@ def test_decode_qwen_heads_long_cache_split_over_many_ctas():
     _decode_case([100000], 28, 4, 128, 3)
 
 
+def test_decode_one_kv_head_more_key_splits_than_one_merge_round_takes():
+    # a single KV head: all CTAs split the same head group's keys (261 splits), more than the 256 the merge fetches in its first round
+    _decode_case([100000], 8, 1, 128, 8)
+
+
 def test_decode_few_long_sequences_one_item_per_cta():
     # unequal long caches whose keys are cut into one item per CTA (the last chunk of every sequence and head is shorter)
     _decode_case([40000, 30001, 20000, 9000], 28, 4, 128, 7, pad=3)
