@@ -239,6 +239,30 @@ def test_attention_tiny_brute_force():
     assert np.allclose(O, ref, rtol=1e-12, atol=1e-13)
 
 
+def test_attention_huge_logits_against_fifty_digit_arithmetic():
+    """Scores hundreds of units apart (what the GPU test with towering keys feeds both sides): the oracle's softmax against the
+    definition evaluated in 60-digit decimal arithmetic, where exp(700) and exp(-700) are ordinary numbers."""
+    from decimal import Decimal, getcontext
+    getcontext().prec = 60
+    g = torch.Generator().manual_seed(31)
+    n, D = 9, 4
+    Q = torch.randn(n, 1, D, generator=g, dtype=torch.float64)
+    K = torch.randn(n, 1, D, generator=g, dtype=torch.float64)
+    V = torch.randn(n, 1, D, generator=g, dtype=torch.float64)
+    K[3:] *= 300.0                       # later keys tower over the first ones, in both directions
+    K[:2] *= 80.0
+    cu = np.array([0, n], dtype=np.int32)
+    O, lse = oc.attention(Q, K, V, cu, scale=0.5)
+    for i in range(n):
+        sc = [Decimal(0.5) * sum(Decimal(float(Q[i, 0, c])) * Decimal(float(K[j, 0, c])) for c in range(D)) for j in range(i + 1)]
+        e = [x.exp() for x in sc]
+        z = sum(e)
+        for c in range(D):
+            want = sum(e[j] / z * Decimal(float(V[j, 0, c])) for j in range(i + 1))
+            assert abs(Decimal(float(O[i, 0, c])) - want) <= Decimal(1e-12) * (1 + abs(want)), (i, c)
+        assert abs(Decimal(float(lse[i, 0])) - z.ln()) <= Decimal(1e-10) * (1 + abs(z.ln())), i
+
+
 def test_attention_closed_forms():
     g = torch.Generator().manual_seed(8)
     n, Hq, Hkv, D = 40, 6, 2, 16
