@@ -256,7 +256,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             ok = all_ok(mbar_wait(bar_s, ph, kWaitCycles));                   // S_j done: the K buffer is free
             if (!ok) break;
             if (j + 1 < nblk) load_kv(sK, &mapK, bar_k, seq_a + (j + 1) * kBN);
-            ok = all_ok(mbar_wait(bar_p0, ph, kWaitCycles) && mbar_wait(bar_v, ph, kWaitCycles));
+            ok = all_ok(mbar_wait(bar_v, ph, kWaitCycles) && mbar_wait(bar_p0, ph, kWaitCycles));
             if (!ok) break;
             if (lane == 0) {
                 tc_fence_after();
@@ -265,19 +265,16 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
                 tc_commit(bar_o0);
             }
-            ok = all_ok(mbar_wait(bar_p1, ph, kWaitCycles));
+            if (j + 1 < nblk) ok = all_ok(mbar_wait(bar_k, (blk0 + j + 1) & 1, kWaitCycles));     // (ahead of the wait for P, as below)
+            ok = ok && all_ok(mbar_wait(bar_p1, ph, kWaitCycles));
             if (!ok) break;
             if (lane == 0) {
                 tc_fence_after();
 #pragma unroll
                 for (int kk = kBN / 32; kk < kBN / 16; ++kk)
                     mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, 1);
+                if (j + 1 < nblk) issue_s();
                 tc_commit(bar_o);
-            }
-            if (j + 1 < nblk) {
-                ok = all_ok(mbar_wait(bar_k, (blk0 + j + 1) & 1, kWaitCycles));
-                if (!ok) break;
-                if (lane == 0) issue_s();
             }
             ok = all_ok(mbar_wait(bar_o, ph, kWaitCycles));                   // PV_j done: the V buffer is free
             if (!ok) break;
@@ -298,7 +295,6 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             mbar_arrive_expect_tx(bar_v, L::kTileBytes);
             for (int c = 0; c < KCH; ++c) tma_load_3d(sV + c * kChunkBytes, &mapV, bar_v, c * 64, kvh, seq_a);
             auto issue_s = [&]() {
-                tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * kChunkBytes + (kk & 3) * 32;
@@ -307,7 +303,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                 tc_commit(bar_s);
             };
             ok = mbar_wait(bar_q, qph, kWaitCycles) && mbar_wait(bar_k, blk0 & 1, kWaitCycles);
-            if (ok) issue_s();
+            if (ok) { tc_fence_after(); issue_s(); }
             for (int j = 0; j < nblk && ok; ++j) {
                 const uint32_t ph = (blk0 + j) & 1;
                 // S_j done: the K buffer is free for the next block
@@ -317,28 +313,29 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     mbar_arrive_expect_tx(bar_k, L::kTileBytes);
                     for (int c = 0; c < KCH; ++c) tma_load_3d(sK + c * kChunkBytes, &mapK, bar_k, c * 64, kvh, seq_a + (j + 1) * kBN);
                 }
-                // O += P_j V_j, started as soon as the first 64 keys of P are in TMEM
-                ok = mbar_wait(bar_p0, ph, kWaitCycles) && mbar_wait(bar_v, ph, kWaitCycles);
+                // O += P_j V_j, started as soon as the first 64 keys of P are in TMEM.  (The waits for the tiles come before the
+                // waits for P: a wait holds this thread for some 70 cycles even when its barrier is complete, and behind a
+                // hand-over of P those cycles are on the chain to the next S.)
+                ok = mbar_wait(bar_v, ph, kWaitCycles) && mbar_wait(bar_p0, ph, kWaitCycles);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < kBN / 32; ++kk)
                     mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
                 tc_commit(bar_o0);                            // for a softmax thread that has to rescale O in the middle of the block
-                ok = mbar_wait(bar_p1, ph, kWaitCycles);
+                if (j + 1 < nblk) ok = mbar_wait(bar_k, (blk0 + j + 1) & 1, kWaitCycles);      // K_{j+1}, asked for at the top of this block
+                ok = ok && mbar_wait(bar_p1, ph, kWaitCycles);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
                 for (int kk = kBN / 32; kk < kBN / 16; ++kk)
                     mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, 1);
-                tc_commit(bar_o);
                 // S_{j+1} goes into the pipe right behind PV_j: tcgen05.mma of one thread execute in issue
-                // order, so PV_j has read P_j before S_{j+1} overwrites the columns they share
-                if (j + 1 < nblk) {
-                    ok = mbar_wait(bar_k, (blk0 + j + 1) & 1, kWaitCycles);
-                    if (!ok) break;
-                    issue_s();
-                }
+                // order, so PV_j has read P_j before S_{j+1} overwrites the columns they share.  The commit that reports PV_j
+                // comes behind the S products (a commit holds this thread as long as a product does, and S_{j+1} is what the
+                // softmax warps wait for): the V buffer is given free that much later, which costs less.
+                if (j + 1 < nblk) issue_s();
+                tc_commit(bar_o);
                 // PV_j done: the V buffer is free
                 ok = mbar_wait(bar_o, ph, kWaitCycles);
                 if (!ok) break;
