@@ -324,7 +324,7 @@ attention_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                     mma_ts(tO, tP + kk * 8, smem_desc_sw128(sV + kk * 2048, kChunkBytes, 1024), idesc_o, (j > 0) || (kk > 0));
                 tc_commit(bar_o0);                            // for a softmax thread that has to rescale O in the middle of the block
                 if (j + 1 < nblk) ok = mbar_wait(bar_k, (blk0 + j + 1) & 1, kWaitCycles);      // K_{j+1}, asked for at the top of this block
-                ok = ok && mbar_wait(bar_p1, ph, kWaitCycles);
+                ok = ok && mbar_poll(bar_p1, ph, kWaitCycles);                                 // polled: what follows is the chain to S_{j+1}
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll

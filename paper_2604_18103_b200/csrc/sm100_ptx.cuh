@@ -45,6 +45,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long lo
     }
     return true;
 }
+// The same wait by polling (mbarrier.test_wait does not suspend the thread): for the one wait of a single thread whose wake-up
+// latency is on a critical chain; it keeps an issue slot of its sub-partition busy while it polls.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_poll(uint32_t bar, uint32_t parity, long long limit_cycles) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (mbar_test_wait(bar, parity)) return true;
+        if (clock64() - t0 > limit_cycles) return false;
+    }
+}
 
 // ---- TMA (tiled loads into this CTA's shared memory) -------------------------
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
