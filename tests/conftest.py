@@ -39,7 +39,7 @@ def pytest_sessionfinish(session, exitstatus):
     if not _ERRORS:
         return
     import json
-    out = os.environ.get("DASH_TEST_RECORD_DIR", os.path.join(ROOT, "gpurun_out"))      # where the session's record goes
+    out = os.environ.get("DASH_TEST_RECORD_DIR", os.path.join(ROOT, "test_records"))      # where the session's record goes
     try:
         os.makedirs(out, exist_ok=True)
         with open(os.path.join(out, "parity_errors.json"), "w") as f:
